@@ -1,0 +1,234 @@
+/*
+ * kvbfp — a KV cache in Block Floating Point (BFP) with K-sort channel
+ * permutation, for NVIDIA B200 (sm_100a).  C ABI; no CUDA or framework types.
+ *
+ * Method: N. Trukhanov, I. Soloveychik, "Accurate Block Quantization in LLMs
+ * with Outliers".  A BFP block is n signed p-bit integer mantissas M_i sharing
+ * one 8-bit exponent e, with values 2^e * M_i (Sec. II-B, Eq. (1)).  Key
+ * channels are reordered once, per head, by a permutation pi found from a
+ * per-channel magnitude statistic (Sec. II-C, Sec. III Algorithm 1); q is
+ * permuted the same way, which leaves q.k unchanged (Eq. (2), (3)).
+ *
+ * Conventions for every call
+ *  - Pointers are DEVICE pointers unless the parameter says "host".  Structs
+ *    (kvbfp_format, kvbfp_cache) live in host memory and are read during the call.
+ *  - The caller owns every buffer.  The library allocates nothing and keeps no
+ *    state between calls except one 4-byte status word per device.
+ *  - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *    default stream) of the CURRENT device; results are valid once the stream
+ *    has been synchronised.
+ *  - Argument errors are found on the host before anything is enqueued and are
+ *    returned as a status.  Data-dependent conditions (non-finite input, a
+ *    position beyond the cache capacity, a sequence longer than the hint) set
+ *    bits in the device status word, skip the offending work, and never trap;
+ *    read them with kvbfp_device_status().
+ *  - Tensors are dense, row-major, last index fastest, 16-byte aligned.
+ *
+ * Storage layout (the paper does not fix one; this is the library's own):
+ *  - mantissa plane  [batch, n_kv_heads, max_seq, row_m] bytes, row_m = head_dim*p/8;
+ *    a row is a little-endian bit stream, stored slot j in bits [j*p, (j+1)*p),
+ *    two's complement (p = 4: low nibble is the even slot);
+ *  - exponent plane  [batch, n_kv_heads, max_seq, row_e] bytes, row_e = head_dim/n;
+ *    byte i belongs to slots [i*n, (i+1)*n) and holds E + 127, where 2^E is the
+ *    largest power of two not above the block's largest magnitude (E >= -127);
+ *    the mantissa's unit weight is 2^(E - (p-2)).  255 is never written.
+ *  - "slot" = position after the permutation: slot j of head h holds original
+ *    channel perm[h*head_dim + j].
+ */
+#ifndef KVBFP_H
+#define KVBFP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KVBFP_OK = 0,
+    KVBFP_ERR_INVALID_ARG = 1,  /* null pointer, bad count, inconsistent sizes          */
+    KVBFP_ERR_UNSUPPORTED = 2,  /* a format or shape the kernels are not built for       */
+    KVBFP_ERR_ALIGNMENT = 3,    /* a pointer that is not 16-byte aligned                 */
+    KVBFP_ERR_CAPACITY = 4,     /* more tokens than the cache holds (host-visible cases) */
+    KVBFP_ERR_WORKSPACE = 5,    /* workspace missing or too small                        */
+    KVBFP_ERR_CUDA = 6          /* a CUDA runtime call or a launch failed                */
+} kvbfp_status;
+
+typedef enum { KVBFP_F32 = 0, KVBFP_BF16 = 1 } kvbfp_dtype;
+typedef enum { KVBFP_STAT_MAXABS = 0, KVBFP_STAT_L2 = 1 } kvbfp_stat;
+
+/* Bits of the device status word. */
+enum {
+    KVBFP_FLAG_NONFINITE = 1u,     /* an input element was Inf or NaN                        */
+    KVBFP_FLAG_POSITION = 2u,      /* start_pos + n_new or seq_len beyond max_seq: skipped   */
+    KVBFP_FLAG_LEN_HINT = 4u,      /* a seq_len exceeded max_len_hint: tokens past it unread */
+    KVBFP_FLAG_WAIT_TIMEOUT = 8u   /* an on-chip copy did not complete within its wait bound */
+};
+
+/* Which decode kernel to run. */
+enum {
+    KVBFP_DECODE_AUTO = 0,  /* the tensor-core kernel                                          */
+    KVBFP_DECODE_SIMT = 1,  /* fp32 FMA on the plain ALUs, one query head at a time            */
+    KVBFP_DECODE_MMA = 2    /* grouped queries as the N operand of warp-level bf16 tensor MMAs */
+};
+/* Optional, or-ed into `flags`: tokens per sequence chunk (a multiple of 128; 0 = chosen by the
+ * library from the batch size and the sequence bound). */
+#define KVBFP_DECODE_CHUNK(tokens) (((uint32_t)(tokens) / 128u) << 8)
+
+/* BFP format and cache geometry (Sec. II-B: block size n, mantissa precision p, b = 8). */
+typedef struct {
+    int32_t batch;
+    int32_t n_kv_heads;
+    int32_t head_dim;   /* 128 */
+    int32_t max_seq;    /* capacity in tokens per (batch, head); a multiple of 16 */
+    int32_t block;      /* n: 16, 32, 64 or 128; divides head_dim */
+    int32_t mant_bits;  /* p: 4, 6 or 8, sign included; mantissas lie in [-(2^(p-1)-1), 2^(p-1)-1] */
+} kvbfp_format;
+
+/* The cache is four caller-owned planes (see "Storage layout"). */
+typedef struct {
+    kvbfp_format fmt;
+    uint8_t* k_mant;
+    uint8_t* k_exp;
+    uint8_t* v_mant;
+    uint8_t* v_exp;
+} kvbfp_cache;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t kvbfp_version(void);
+
+/* Text of a status code (static storage, never NULL). */
+const char* kvbfp_status_string(kvbfp_status s);
+
+/* Text of the last CUDA error seen by this thread inside the library (thread-local storage;
+ * empty string if none). */
+const char* kvbfp_last_cuda_error(void);
+
+/* Sizes in bytes of ONE mantissa plane and ONE exponent plane of `fmt` (host pointers out).
+ * Bits per stored element are p + 8/n (Sec. III: BFP12 = 4-bit mantissas + the shared byte). */
+kvbfp_status kvbfp_plane_bytes(const kvbfp_format* fmt, size_t* mant_bytes, size_t* exp_bytes);
+
+/*
+ * K-sort, Algorithm 1 steps 1-2 (Sec. III), run once before inference.
+ *   x            [n_tokens, n_heads, head_dim] of `dt`: calibration keys, or W_k transposed so
+ *                that the reduced axis comes first
+ *   stat         KVBFP_STAT_MAXABS: stat[h,c] = max_t |x[t,h,c]|   (exact)
+ *                KVBFP_STAT_L2:     stat[h,c] = sqrt(sum_t x^2), summed in fp64 (Algorithm 1 step 1)
+ *   stat_out     [n_heads*head_dim] f32, required
+ *   perm_out     [n_heads*head_dim] i32: slot j of head h holds channel perm_out[h*d+j]; ascending
+ *                statistic, equal statistics in channel order (stable)
+ *   inv_perm_out [n_heads*head_dim] i32 or NULL: inv_perm[h*d + perm[h*d+j]] = j
+ *   workspace    KVBFP_STAT_L2 only: n_heads*head_dim*8 bytes for the fp64 sums; NULL for MAXABS
+ * Non-finite inputs set KVBFP_FLAG_NONFINITE; the permutation is then unspecified but valid.
+ */
+kvbfp_status kvbfp_calibrate(const void* x, kvbfp_dtype dt, int64_t n_tokens, int32_t n_heads,
+                             int32_t head_dim, kvbfp_stat stat, float* stat_out, int32_t* perm_out,
+                             int32_t* inv_perm_out, void* workspace, size_t workspace_bytes,
+                             void* stream);
+
+/*
+ * Algorithm 1 steps 3-4: fold a permutation into a projection weight, once, offline.
+ *   w   [n_heads*head_dim, d_in] of `dt` (rows = output channels of W_k or W_q)
+ *   out [n_heads*head_dim, d_in] of `dt`, out[h*d + j, :] = w[h*d + perm[h*d+j], :]; out != w
+ * With folded weights the run-time gathers are not needed: pass perm_k = NULL to append/decode.
+ */
+kvbfp_status kvbfp_fold_perm(const void* w, kvbfp_dtype dt, int32_t n_heads, int32_t head_dim,
+                             int64_t d_in, const int32_t* perm, void* out, void* stream);
+
+/*
+ * Cache write (Sec. II-A; Sec. III par. 2): permute each new row, take the shared exponent of each
+ * block from its largest magnitude, round mantissas to nearest (ties to even), clamp to the
+ * symmetric range, pack, store (Sec. II-B last paragraph).
+ *   k_new, v_new [batch, n_new, n_kv_heads, head_dim] of `dt`; either may be NULL (plane untouched)
+ *   start_pos    [batch] i32: row t of sequence b goes to position start_pos[b] + t
+ *   perm_k/v     [n_kv_heads*head_dim] i32 or NULL (identity, e.g. when folded into the weights)
+ * A sequence whose rows would pass max_seq is skipped whole and sets KVBFP_FLAG_POSITION.
+ */
+kvbfp_status kvbfp_append(const kvbfp_cache* cache, const void* k_new, const void* v_new,
+                          kvbfp_dtype dt, int32_t n_new, const int32_t* start_pos,
+                          const int32_t* perm_k, const int32_t* perm_v, void* stream);
+
+/*
+ * Eq. (1): rows [t0, t0+n_tok) of (b, h) of one plane pair back to numbers (exact in f32 and bf16).
+ *   perm  NULL: out[t, j] = slot j;  else out[t, perm[h*d+j]] = slot j (original channel order)
+ *   out   [n_tok, head_dim] of out_dt
+ */
+kvbfp_status kvbfp_dequant(const kvbfp_format* fmt, const uint8_t* mant, const uint8_t* exp8,
+                           int32_t b, int32_t h, int32_t t0, int32_t n_tok, const int32_t* perm,
+                           void* out, kvbfp_dtype out_dt, void* stream);
+
+/* Bytes of workspace kvbfp_decode_attn needs for this cache geometry (0 on invalid arguments). */
+size_t kvbfp_decode_workspace_bytes(const kvbfp_format* fmt, int32_t n_q_heads);
+
+/*
+ * One decode step of attention read straight from the packed cache (Sec. II-A; Sec. III par. 2:
+ * keys are read back and multiplied with pi(q)): scores = scale * pi(q).K^T over tokens
+ * t < seq_lens[b], softmax, times V; K/V are dequantised in registers, never written back.
+ *   q              [batch, n_q_heads, head_dim] of q_dt, original channel order
+ *   n_q_heads      multiple of n_kv_heads; query head hq reads KV head hq / (n_q_heads/n_kv_heads)
+ *   seq_lens       [batch] i32
+ *   max_len_hint   host-known upper bound of seq_lens (0 = max_seq); sizes the launch only
+ *   perm_k         permutation the keys were appended with (NULL = identity); q is gathered by it
+ *   inv_perm_v     inverse of the permutation V was appended with (NULL = identity):
+ *                  out[c] = o_slot[inv_perm_v[g*d + c]]
+ *   softmax_scale  0 means 1/sqrt(head_dim)
+ *   q_mant_bits    0: q used as given.  8: pi(q) is first cast to BFP with 8-bit mantissas and the
+ *                  cache's block size (the BFP16 query of Sec. IV)
+ *   out            [batch, n_q_heads, head_dim] f32; zeros where seq_lens[b] == 0
+ *   workspace      at least kvbfp_decode_workspace_bytes() bytes, contents need no initialisation
+ *   flags          KVBFP_DECODE_* [| KVBFP_DECODE_CHUNK(tokens)]
+ * The sequence is split into chunks handled independently; a second kernel merges the per-chunk
+ * (max, sum, output) triples with log-sum-exp weights.
+ */
+kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt,
+                               int32_t n_q_heads, const int32_t* seq_lens, int32_t max_len_hint,
+                               const int32_t* perm_k, const int32_t* inv_perm_v,
+                               float softmax_scale, int32_t q_mant_bits, float* out,
+                               void* workspace, size_t workspace_bytes, uint32_t flags,
+                               void* stream);
+
+/*
+ * One whole decode step for a caller whose new token lives in HOST memory (Sec. II-A: per step only
+ * the new token's q, k, v are computed; the rest is read from the cache): copies k_new, v_new and q
+ * to the device, appends the token (kvbfp_append with n_new = 1), runs kvbfp_decode_attn, copies the
+ * result back and synchronises `stream`, so out_host is valid on return.
+ *   k_new_host, v_new_host  host [batch, 1, n_kv_heads, head_dim] of `dt` (pinned memory lets the
+ *                           copies run asynchronously)
+ *   q_host                  host [batch, n_q_heads, head_dim] of `dt`
+ *   out_host                host [batch, n_q_heads, head_dim] f32
+ *   start_pos, seq_lens     device [batch] i32, as in kvbfp_append / kvbfp_decode_attn
+ *   staging                 device scratch of at least kvbfp_step_staging_bytes() bytes
+ * All other parameters as in kvbfp_append and kvbfp_decode_attn.
+ */
+size_t kvbfp_step_staging_bytes(const kvbfp_format* fmt, int32_t n_q_heads, kvbfp_dtype dt);
+kvbfp_status kvbfp_decode_step_host(const kvbfp_cache* cache, const void* k_new_host,
+                                    const void* v_new_host, const void* q_host, kvbfp_dtype dt,
+                                    int32_t n_q_heads, const int32_t* start_pos,
+                                    const int32_t* seq_lens, int32_t max_len_hint,
+                                    const int32_t* perm_k, const int32_t* perm_v,
+                                    const int32_t* inv_perm_v, float softmax_scale,
+                                    float* out_host, void* staging, size_t staging_bytes,
+                                    void* workspace, size_t workspace_bytes, uint32_t flags,
+                                    void* stream);
+
+/*
+ * Profiling aid.  After this call, every kvbfp_decode_attn issued from the calling thread records
+ * `start_event` just before and `stop_event` just after its main kernel (the one that streams the
+ * cache), on the call's stream.  Both are cudaEvent_t passed as void*; (NULL, NULL) switches it off.
+ */
+kvbfp_status kvbfp_profile_decode_events(void* start_event, void* stop_event);
+
+/*
+ * Synchronises `stream`, copies the device status word of the current device to *flags_out (host
+ * pointer) and clears it.
+ */
+kvbfp_status kvbfp_device_status(uint32_t* flags_out, void* stream);
+
+/* Number of kernels the library has launched from this process so far (all devices). */
+uint64_t kvbfp_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVBFP_H */

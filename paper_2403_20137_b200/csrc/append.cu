@@ -1,0 +1,212 @@
+// Cache write: permute, shared exponent, round, clamp, pack, store (Sec. II-B last paragraph,
+// Sec. III par. 2 of the paper; Algorithm 1 step 3 applied at run time as a gather).
+//
+// Sixteen lanes own one (token, head) row of 128 channels, eight stored slots per lane, so a warp
+// writes two rows per step.  A block of n slots is held by n/8 neighbouring lanes; its largest
+// magnitude is found with xor-shuffles on the IEEE bit patterns (integer compare = exact).
+#include "common.cuh"
+
+namespace kvbfp {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kRowsPerCta = kThreads / 16;
+
+struct AppendArgs {
+    const void* src[2];      // k_new, v_new (nullptr = skip)
+    uint8_t* mant[2];
+    uint8_t* exp8[2];
+    const int32_t* perm[2];
+    const int32_t* start_pos;
+    int32_t batch, n_new, n_heads, max_seq;
+    uint32_t* status;
+};
+
+template <typename T>
+__device__ __forceinline__ void load8(const T* p, float (&v)[8]);
+
+template <>
+__device__ __forceinline__ void load8<float>(const float* p, float (&v)[8]) {
+    float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+template <>
+__device__ __forceinline__ void load8<__nv_bfloat16>(const __nv_bfloat16* p, float (&v)[8]) {
+    uint4 a = __ldg(reinterpret_cast<const uint4*>(p));
+    uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        v[2 * i] = __uint_as_float(w[i] << 16);
+        v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+}
+
+template <int P, int N, typename T>
+__global__ void __launch_bounds__(kThreads) append_quant_pack(AppendArgs a) {
+    constexpr int D = kHeadDim;
+    constexpr int ROW_M = D * P / 8, ROW_E = D / N;
+    constexpr int LANES_PER_BLOCK = N / 8;
+    constexpr int QMAX = (1 << (P - 1)) - 1;
+    __shared__ float stage[kRowsPerCta][D];
+
+    const int which = blockIdx.y;
+    const T* src = static_cast<const T*>(a.src[which]);
+    if (!src) return;
+    const int32_t* perm = a.perm[which];
+    const int sub = threadIdx.x & 15;          // lane within the row
+    const int rloc = threadIdx.x >> 4;         // row within the CTA
+    const int64_t n_rows = (int64_t)a.batch * a.n_new * a.n_heads;
+
+    for (int64_t r0 = (int64_t)blockIdx.x * kRowsPerCta; r0 < n_rows; r0 += (int64_t)gridDim.x * kRowsPerCta) {
+        const int64_t r = r0 + rloc;
+        const bool live = r < n_rows;
+        float v[8];
+        int h = 0, b = 0, t = 0;
+        if (live) {
+            h = (int)(r % a.n_heads);
+            int64_t bt = r / a.n_heads;
+            t = (int)(bt % a.n_new);
+            b = (int)(bt / a.n_new);
+            load8<T>(src + r * D + sub * 8, v);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        }
+        if (perm) {   // Algorithm 1 step 3: slot j takes channel perm[h][j]
+#pragma unroll
+            for (int i = 0; i < 8; ++i) stage[rloc][sub * 8 + i] = v[i];
+            __syncwarp();
+            if (live) {
+                const int4* pp = reinterpret_cast<const int4*>(perm + h * D + sub * 8);
+                int4 p0 = __ldg(pp), p1 = __ldg(pp + 1);
+                int idx[8] = {p0.x, p0.y, p0.z, p0.w, p1.x, p1.y, p1.z, p1.w};
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = stage[rloc][idx[i] & (D - 1)];
+            }
+            __syncwarp();
+        }
+        // shared exponent: the biased exponent field of the block's largest magnitude
+        uint32_t amax = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) amax = max(amax, __float_as_uint(v[i]) & 0x7fffffffu);
+#pragma unroll
+        for (int off = 1; off < LANES_PER_BLOCK; off <<= 1)
+            amax = max(amax, __shfl_xor_sync(0xffffffffu, amax, off));
+        int e8 = (int)(amax >> 23);
+        if (e8 == 255) {            // Inf or NaN somewhere in the block
+            if (live) raise_flag(a.status, KVBFP_FLAG_NONFINITE);
+            e8 = 254;
+        }
+        // t = x * 2^(127 - e8 + p - 2), applied as two exact power-of-two factors
+        const int k = 127 - e8 + (P - 2);
+        const int k1 = k >> 1, k2 = k - k1;
+        const float s1 = pow2i(k1), s2 = pow2i(k2);
+        int m[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float tv = (v[i] * s1) * s2;
+            tv = fminf(fmaxf(tv, (float)-QMAX), (float)QMAX);   // NaN -> -QMAX..QMAX, stays in range
+            m[i] = __float2int_rn(tv);                           // to nearest, ties to even
+        }
+        if (!live) continue;
+        const int sp = a.start_pos[b];
+        if (sp < 0 || (int64_t)sp + a.n_new > a.max_seq) {
+            if (t == 0 && h == 0 && sub == 0) raise_flag(a.status, KVBFP_FLAG_POSITION);
+            continue;
+        }
+        const int64_t pos = ((int64_t)b * a.n_heads + h) * a.max_seq + sp + t;
+        uint8_t* mrow = a.mant[which] + pos * ROW_M;
+        if (P == 4) {
+            uint32_t w = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w |= ((uint32_t)m[i] & 0xfu) << (4 * i);
+            reinterpret_cast<uint32_t*>(mrow)[sub] = w;
+        } else if (P == 6) {
+            uint64_t w = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) w |= ((uint64_t)((uint32_t)m[i] & 0x3fu)) << (6 * i);
+            uint16_t* o = reinterpret_cast<uint16_t*>(mrow + sub * 6);
+            o[0] = (uint16_t)w;
+            o[1] = (uint16_t)(w >> 16);
+            o[2] = (uint16_t)(w >> 32);
+        } else {
+            uint32_t lo = 0, hi = 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                lo |= ((uint32_t)m[i] & 0xffu) << (8 * i);
+                hi |= ((uint32_t)m[i + 4] & 0xffu) << (8 * i);
+            }
+            reinterpret_cast<uint2*>(mrow)[sub] = make_uint2(lo, hi);
+        }
+        if ((sub % LANES_PER_BLOCK) == 0) a.exp8[which][pos * ROW_E + sub / LANES_PER_BLOCK] = (uint8_t)e8;
+    }
+}
+
+template <int P, int N, typename T>
+kvbfp_status launch(const AppendArgs& a, int64_t n_rows, cudaStream_t s) {
+    int64_t want = (n_rows + kRowsPerCta - 1) / kRowsPerCta;
+    int gx = (int)(want < 148 * 32 ? want : 148 * 32);
+    dim3 grid(gx, 2);
+    append_quant_pack<P, N, T><<<grid, kThreads, 0, s>>>(a);
+    KVBFP_LAUNCH_CHECK("append_quant_pack");
+    return KVBFP_OK;
+}
+
+template <int P, typename T>
+kvbfp_status launch_n(int n, const AppendArgs& a, int64_t n_rows, cudaStream_t s) {
+    switch (n) {
+        case 16: return launch<P, 16, T>(a, n_rows, s);
+        case 32: return launch<P, 32, T>(a, n_rows, s);
+        case 64: return launch<P, 64, T>(a, n_rows, s);
+        case 128: return launch<P, 128, T>(a, n_rows, s);
+    }
+    return KVBFP_ERR_UNSUPPORTED;
+}
+
+template <typename T>
+kvbfp_status launch_p(int p, int n, const AppendArgs& a, int64_t n_rows, cudaStream_t s) {
+    switch (p) {
+        case 4: return launch_n<4, T>(n, a, n_rows, s);
+        case 6: return launch_n<6, T>(n, a, n_rows, s);
+        case 8: return launch_n<8, T>(n, a, n_rows, s);
+    }
+    return KVBFP_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+}  // namespace kvbfp
+
+extern "C" kvbfp_status kvbfp_append(const kvbfp_cache* cache, const void* k_new, const void* v_new,
+                                     kvbfp_dtype dt, int32_t n_new, const int32_t* start_pos,
+                                     const int32_t* perm_k, const int32_t* perm_v, void* stream) {
+    using namespace kvbfp;
+    if (!cache) return KVBFP_ERR_INVALID_ARG;
+    kvbfp_status st = check_format(&cache->fmt);
+    if (st != KVBFP_OK) return st;
+    if (!start_pos || n_new < 0 || (!k_new && !v_new)) return KVBFP_ERR_INVALID_ARG;
+    if (dt != KVBFP_F32 && dt != KVBFP_BF16) return KVBFP_ERR_INVALID_ARG;
+    if (k_new && (!cache->k_mant || !cache->k_exp)) return KVBFP_ERR_INVALID_ARG;
+    if (v_new && (!cache->v_mant || !cache->v_exp)) return KVBFP_ERR_INVALID_ARG;
+    if (n_new > cache->fmt.max_seq) return KVBFP_ERR_CAPACITY;
+    const void* ptrs[] = {k_new, v_new, cache->k_mant, cache->k_exp, cache->v_mant, cache->v_exp, perm_k, perm_v};
+    for (const void* p : ptrs)
+        if (p && !aligned16(p)) return KVBFP_ERR_ALIGNMENT;
+    if (n_new == 0) return KVBFP_OK;
+
+    AppendArgs a;
+    a.src[0] = k_new; a.src[1] = v_new;
+    a.mant[0] = cache->k_mant; a.mant[1] = cache->v_mant;
+    a.exp8[0] = cache->k_exp; a.exp8[1] = cache->v_exp;
+    a.perm[0] = perm_k; a.perm[1] = perm_v;
+    a.start_pos = start_pos;
+    a.batch = cache->fmt.batch; a.n_new = n_new; a.n_heads = cache->fmt.n_kv_heads;
+    a.max_seq = cache->fmt.max_seq;
+    st = status_word(&a.status);
+    if (st != KVBFP_OK) return st;
+    const int64_t n_rows = (int64_t)a.batch * n_new * a.n_heads;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (dt == KVBFP_F32) return launch_p<float>(cache->fmt.mant_bits, cache->fmt.block, a, n_rows, s);
+    return launch_p<__nv_bfloat16>(cache->fmt.mant_bits, cache->fmt.block, a, n_rows, s);
+}

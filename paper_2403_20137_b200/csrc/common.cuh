@@ -1,0 +1,73 @@
+// Shared host/device helpers of the kvbfp CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "kvbfp.h"
+
+namespace kvbfp {
+
+constexpr int kHeadDim = 128;
+
+// ---- host side -------------------------------------------------------------
+
+// Records a failed CUDA call for kvbfp_last_cuda_error() and maps it to a status.
+kvbfp_status cuda_fail(cudaError_t e, const char* what);
+// Address of the device status word of the current device (no allocation: a __device__ symbol).
+kvbfp_status status_word(uint32_t** ptr);
+void count_launch(int n = 1);
+
+#define KVBFP_CUDA(call)                                                         \
+    do {                                                                         \
+        cudaError_t e__ = (call);                                                \
+        if (e__ != cudaSuccess) return ::kvbfp::cuda_fail(e__, #call);           \
+    } while (0)
+
+#define KVBFP_LAUNCH_CHECK(name)                                                 \
+    do {                                                                         \
+        cudaError_t e__ = cudaGetLastError();                                    \
+        if (e__ != cudaSuccess) return ::kvbfp::cuda_fail(e__, name);            \
+        ::kvbfp::count_launch();                                                 \
+    } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+inline kvbfp_status check_format(const kvbfp_format* f) {
+    if (!f) return KVBFP_ERR_INVALID_ARG;
+    if (f->batch < 1 || f->n_kv_heads < 1 || f->max_seq < 1) return KVBFP_ERR_INVALID_ARG;
+    if (f->head_dim != kHeadDim) return KVBFP_ERR_UNSUPPORTED;
+    if (f->block != 16 && f->block != 32 && f->block != 64 && f->block != 128) return KVBFP_ERR_UNSUPPORTED;
+    if (f->mant_bits != 4 && f->mant_bits != 6 && f->mant_bits != 8) return KVBFP_ERR_UNSUPPORTED;
+    if (f->max_seq % 16 != 0) return KVBFP_ERR_INVALID_ARG;
+    return KVBFP_OK;
+}
+inline size_t row_m_bytes(const kvbfp_format& f) { return (size_t)f.head_dim * f.mant_bits / 8; }
+inline size_t row_e_bytes(const kvbfp_format& f) { return (size_t)(f.head_dim / f.block); }
+
+// ---- device side -----------------------------------------------------------
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
+
+// 2^k for k in [-126, 127]
+__device__ __forceinline__ float pow2i(int k) { return __uint_as_float((uint32_t)(k + 127) << 23); }
+
+// Weight of one mantissa unit, 2^(e8 - 127 - (p-2)), as an fp32 number; exact down to 2^-133
+// (subnormal) for e8 = 0, p = 8.
+__device__ __forceinline__ float unit_weight(int e8, int p) {
+    int f = e8 - (p - 2);                 // biased exponent field of the result
+    return f >= 1 ? __uint_as_float((uint32_t)f << 23) : __uint_as_float(1u << (22 + f));
+}
+
+__device__ __forceinline__ void raise_flag(uint32_t* status, uint32_t bit) { atomicOr(status, bit); }
+
+// Sign-extended p-bit field starting at bit `bit` of a little-endian byte row.
+__device__ __forceinline__ int extract_field(const uint8_t* row, int bit, int p) {
+    int byte = bit >> 3, sh = bit & 7;
+    uint32_t w = row[byte] | ((uint32_t)row[byte + ((sh + p > 8) ? 1 : 0)] << 8);
+    int v = (int)((w >> sh) & ((1u << p) - 1u));
+    return (v ^ (1 << (p - 1))) - (1 << (p - 1));
+}
+
+}  // namespace kvbfp

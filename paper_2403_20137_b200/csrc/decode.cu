@@ -1,0 +1,198 @@
+// Decode-attention entry point: argument checks, sequence chunking, and the log-sum-exp merge of the
+// per-chunk partial results (the split over sequence length).
+#include <math.h>
+
+#include "decode.cuh"
+
+namespace kvbfp {
+namespace {
+
+// One warp per (batch, query head): out = sum_i 2^(m_i - m) o_i / sum_i 2^(m_i - m) l_i.
+__global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ partials, const int32_t* __restrict__ seq_lens,
+                                                 const int32_t* __restrict__ inv_perm_v, float* __restrict__ out,
+                                                 int n_rows, int n_q_heads, int group, int n_chunks, int chunk,
+                                                 int len_cap) {
+    constexpr int D = kHeadDim;
+    __shared__ float so[4][D];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = blockIdx.x * 4 + warp;           // b * Hq + hq
+    if (row >= n_rows) return;
+    const int b = row / n_q_heads, hq = row % n_q_heads;
+    int len = seq_lens[b];
+    len = len < 0 ? 0 : (len > len_cap ? len_cap : len);
+    const int nc = (len + chunk - 1) / chunk;        // chunks that hold tokens
+    const float* base = partials + (int64_t)row * n_chunks * kPartStride;
+    float m = -INFINITY;
+    for (int i = lane; i < nc; i += 32) m = fmaxf(m, base[(int64_t)i * kPartStride + D]);
+#pragma unroll
+    for (int off = 16; off; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float l = 0.f;
+    for (int i = 0; i < nc; ++i) {
+        const float* p = base + (int64_t)i * kPartStride;
+        const float w = exp2f(p[D] - m);
+        const float4 o = *reinterpret_cast<const float4*>(p + lane * 4);
+        acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+        l += w * p[D + 1];
+    }
+    const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
+    float* dst = out + (int64_t)row * D;
+    if (!inv_perm_v) {
+        *reinterpret_cast<float4*>(dst + lane * 4) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+    } else {
+        so[warp][lane * 4 + 0] = acc.x * inv; so[warp][lane * 4 + 1] = acc.y * inv;
+        so[warp][lane * 4 + 2] = acc.z * inv; so[warp][lane * 4 + 3] = acc.w * inv;
+        __syncwarp();
+        const int32_t* ip = inv_perm_v + (hq / group) * D;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) dst[lane + 32 * k] = so[warp][ip[lane + 32 * k] & (D - 1)];
+    }
+}
+
+inline int max_chunks(const kvbfp_format& f) { return (f.max_seq + kMinChunk - 1) / kMinChunk; }
+
+thread_local cudaEvent_t t_ev_start = nullptr, t_ev_stop = nullptr;
+
+}  // namespace
+
+void profile_events(cudaEvent_t* start, cudaEvent_t* stop) {
+    *start = t_ev_start;
+    *stop = t_ev_stop;
+}
+
+size_t qfrag_bytes(const kvbfp_format& f, int n_q_heads) {
+    const int group = n_q_heads / f.n_kv_heads;
+    const int nt = (group + 3) / 4;                  // four query heads per 8-column MMA tile
+    return (size_t)f.batch * f.n_kv_heads * nt * 8 * 32 * 2 * sizeof(uint32_t);
+}
+
+}  // namespace kvbfp
+
+extern "C" size_t kvbfp_decode_workspace_bytes(const kvbfp_format* fmt, int32_t n_q_heads) {
+    using namespace kvbfp;
+    if (check_format(fmt) != KVBFP_OK || n_q_heads < 1 || n_q_heads % fmt->n_kv_heads != 0) return 0;
+    size_t part = (size_t)fmt->batch * n_q_heads * max_chunks(*fmt) * kPartStride * sizeof(float);
+    return qfrag_bytes(*fmt, n_q_heads) + part;
+}
+
+extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt,
+                                          int32_t n_q_heads, const int32_t* seq_lens, int32_t max_len_hint,
+                                          const int32_t* perm_k, const int32_t* inv_perm_v, float softmax_scale,
+                                          int32_t q_mant_bits, float* out, void* workspace, size_t workspace_bytes,
+                                          uint32_t flags, void* stream) {
+    using namespace kvbfp;
+    if (!cache) return KVBFP_ERR_INVALID_ARG;
+    const kvbfp_format& f = cache->fmt;
+    kvbfp_status st = check_format(&f);
+    if (st != KVBFP_OK) return st;
+    if (!cache->k_mant || !cache->k_exp || !cache->v_mant || !cache->v_exp || !q || !seq_lens || !out)
+        return KVBFP_ERR_INVALID_ARG;
+    if (n_q_heads < 1 || n_q_heads % f.n_kv_heads != 0) return KVBFP_ERR_INVALID_ARG;
+    const int group = n_q_heads / f.n_kv_heads;
+    if (group > 8) return KVBFP_ERR_UNSUPPORTED;
+    if (q_dt != KVBFP_F32 && q_dt != KVBFP_BF16) return KVBFP_ERR_INVALID_ARG;
+    if (q_mant_bits != 0 && q_mant_bits != 8) return KVBFP_ERR_UNSUPPORTED;
+    if (max_len_hint < 0 || !(softmax_scale >= 0.f) || isinf(softmax_scale)) return KVBFP_ERR_INVALID_ARG;
+    const uint32_t impl = flags & 0xffu, chunk_units = (flags >> 8) & 0xfffu;
+    if (impl > KVBFP_DECODE_MMA || (flags >> 20)) return KVBFP_ERR_INVALID_ARG;
+    const void* ptrs[] = {cache->k_mant, cache->k_exp, cache->v_mant, cache->v_exp, q, out, workspace, perm_k, inv_perm_v};
+    for (const void* p : ptrs)
+        if (p && !aligned16(p)) return KVBFP_ERR_ALIGNMENT;
+    const size_t need = kvbfp_decode_workspace_bytes(&f, n_q_heads);
+    if (!workspace || workspace_bytes < need) return KVBFP_ERR_WORKSPACE;
+
+    DecodeArgs a;
+    a.fmt = f;
+    a.k_mant = cache->k_mant; a.k_exp = cache->k_exp; a.v_mant = cache->v_mant; a.v_exp = cache->v_exp;
+    a.q = q; a.q_is_bf16 = (q_dt == KVBFP_BF16); a.n_q_heads = n_q_heads;
+    a.seq_lens = seq_lens; a.perm_k = perm_k; a.inv_perm_v = inv_perm_v;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)f.head_dim);
+    a.scale_log2e = scale * 1.4426950408889634f;
+    a.q_mant_bits = q_mant_bits;
+    a.out = out;
+    a.qfrag = static_cast<uint32_t*>(workspace);
+    a.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + qfrag_bytes(f, n_q_heads));
+    a.len_cap = (max_len_hint > 0 && max_len_hint < f.max_seq) ? max_len_hint : f.max_seq;
+
+    // Sequence chunking: enough independent (batch, kv head, chunk) items to keep every warp slot of
+    // the machine busy for a few rounds, chunks in multiples of kMinChunk tokens.
+    int chunk;
+    if (chunk_units) {
+        chunk = (int)chunk_units * kMinChunk;
+    } else {
+        const int64_t pairs = (int64_t)f.batch * f.n_kv_heads;
+        const int64_t target_items = 148 * 16 * 4;
+        int64_t want = (target_items + pairs - 1) / pairs;
+        if (want < 1) want = 1;
+        int64_t per = (a.len_cap + want - 1) / want;
+        chunk = (int)(((per + kMinChunk - 1) / kMinChunk) * kMinChunk);
+        if (chunk < kMinChunk) chunk = kMinChunk;
+    }
+    a.chunk = chunk;
+    a.n_chunks = (a.len_cap + chunk - 1) / chunk;
+    st = status_word(&a.status);
+    if (st != KVBFP_OK) return st;
+
+    cudaStream_t s = (cudaStream_t)stream;
+    st = (impl == KVBFP_DECODE_SIMT) ? launch_decode_simt(a, s) : launch_decode_mma(a, s);
+    if (st != KVBFP_OK) return st;
+    const int n_rows = f.batch * n_q_heads;
+    lse_merge<<<(n_rows + 3) / 4, 128, 0, s>>>(a.partials, seq_lens, inv_perm_v, out, n_rows, n_q_heads, group,
+                                              a.n_chunks, a.chunk, a.len_cap);
+    KVBFP_LAUNCH_CHECK("lse_merge");
+    return KVBFP_OK;
+}
+
+extern "C" kvbfp_status kvbfp_profile_decode_events(void* start_event, void* stop_event) {
+    if ((start_event == nullptr) != (stop_event == nullptr)) return KVBFP_ERR_INVALID_ARG;
+    kvbfp::t_ev_start = (cudaEvent_t)start_event;
+    kvbfp::t_ev_stop = (cudaEvent_t)stop_event;
+    return KVBFP_OK;
+}
+
+extern "C" size_t kvbfp_step_staging_bytes(const kvbfp_format* fmt, int32_t n_q_heads, kvbfp_dtype dt) {
+    using namespace kvbfp;
+    if (check_format(fmt) != KVBFP_OK || n_q_heads < 1 || (dt != KVBFP_F32 && dt != KVBFP_BF16)) return 0;
+    const size_t es = dt == KVBFP_F32 ? 4 : 2;
+    const size_t kv = (size_t)fmt->batch * fmt->n_kv_heads * fmt->head_dim * es;
+    const size_t qb = (size_t)fmt->batch * n_q_heads * fmt->head_dim * es;
+    const size_t ob = (size_t)fmt->batch * n_q_heads * fmt->head_dim * sizeof(float);
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    return up(kv) * 2 + up(qb) + up(ob);
+}
+
+extern "C" kvbfp_status kvbfp_decode_step_host(const kvbfp_cache* cache, const void* k_new_host,
+                                               const void* v_new_host, const void* q_host, kvbfp_dtype dt,
+                                               int32_t n_q_heads, const int32_t* start_pos, const int32_t* seq_lens,
+                                               int32_t max_len_hint, const int32_t* perm_k, const int32_t* perm_v,
+                                               const int32_t* inv_perm_v, float softmax_scale, float* out_host,
+                                               void* staging, size_t staging_bytes, void* workspace,
+                                               size_t workspace_bytes, uint32_t flags, void* stream) {
+    using namespace kvbfp;
+    if (!cache || !k_new_host || !v_new_host || !q_host || !out_host || !start_pos || !seq_lens)
+        return KVBFP_ERR_INVALID_ARG;
+    const size_t need = kvbfp_step_staging_bytes(&cache->fmt, n_q_heads, dt);
+    if (need == 0) return KVBFP_ERR_INVALID_ARG;
+    if (!staging || staging_bytes < need) return KVBFP_ERR_WORKSPACE;
+    if (!aligned16(staging)) return KVBFP_ERR_ALIGNMENT;
+    const kvbfp_format& f = cache->fmt;
+    const size_t es = dt == KVBFP_F32 ? 4 : 2;
+    const size_t kv = (size_t)f.batch * f.n_kv_heads * f.head_dim * es;
+    const size_t qb = (size_t)f.batch * n_q_heads * f.head_dim * es;
+    const size_t ob = (size_t)f.batch * n_q_heads * f.head_dim * sizeof(float);
+    auto up = [](size_t x) { return (x + 255) & ~(size_t)255; };
+    uint8_t* base = static_cast<uint8_t*>(staging);
+    uint8_t *dk = base, *dv = base + up(kv), *dq = base + 2 * up(kv), *dout = base + 2 * up(kv) + up(qb);
+    cudaStream_t s = (cudaStream_t)stream;
+    KVBFP_CUDA(cudaMemcpyAsync(dk, k_new_host, kv, cudaMemcpyHostToDevice, s));
+    KVBFP_CUDA(cudaMemcpyAsync(dv, v_new_host, kv, cudaMemcpyHostToDevice, s));
+    KVBFP_CUDA(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));
+    kvbfp_status st = kvbfp_append(cache, dk, dv, dt, 1, start_pos, perm_k, perm_v, stream);
+    if (st != KVBFP_OK) return st;
+    st = kvbfp_decode_attn(cache, dq, dt, n_q_heads, seq_lens, max_len_hint, perm_k, inv_perm_v, softmax_scale, 0,
+                           reinterpret_cast<float*>(dout), workspace, workspace_bytes, flags, stream);
+    if (st != KVBFP_OK) return st;
+    KVBFP_CUDA(cudaMemcpyAsync(out_host, dout, ob, cudaMemcpyDeviceToHost, s));
+    KVBFP_CUDA(cudaStreamSynchronize(s));
+    return KVBFP_OK;
+}

@@ -1,0 +1,38 @@
+// Internal interface between the decode entry point and its kernels.
+#pragma once
+#include "common.cuh"
+
+namespace kvbfp {
+
+// One partial result per (batch, query head, chunk): PSTRIDE floats =
+// o[128] (sum of 2^(s-m) * V over the chunk, stored-slot order), m (running max, log2 units), l (sum).
+constexpr int kPartStride = kHeadDim + 4;
+constexpr int kMinChunk = 128;     // tokens; chunk sizes are multiples of this
+
+struct DecodeArgs {
+    kvbfp_format fmt;
+    const uint8_t *k_mant, *k_exp, *v_mant, *v_exp;
+    const void* q;            // [B, Hq, d]
+    int q_is_bf16;
+    int n_q_heads;
+    const int32_t* seq_lens;
+    const int32_t* perm_k;
+    const int32_t* inv_perm_v;
+    float scale_log2e;        // softmax scale * log2(e)
+    int q_mant_bits;
+    float* out;
+    uint32_t* qfrag;          // workspace region for the tensor-core kernel's B fragments
+    float* partials;          // workspace region [B, Hq, n_chunks, kPartStride]
+    int chunk;                // tokens per chunk
+    int n_chunks;
+    int len_cap;              // min(max_len_hint, max_seq)
+    uint32_t* status;
+};
+
+kvbfp_status launch_decode_simt(const DecodeArgs& a, cudaStream_t s);
+kvbfp_status launch_decode_mma(const DecodeArgs& a, cudaStream_t s);
+size_t qfrag_bytes(const kvbfp_format& f, int n_q_heads);
+// Events the caller asked to have recorded around the main decode kernel (nullptr = none).
+void profile_events(cudaEvent_t* start, cudaEvent_t* stop);
+
+}  // namespace kvbfp

@@ -1,0 +1,83 @@
+// Library-wide host state: status word address, error text, launch counter, small queries.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+
+#include "common.cuh"
+
+namespace kvbfp {
+
+// One status word per device: a __device__ symbol, so nothing is allocated.
+__device__ uint32_t g_status_word = 0;
+
+static thread_local char t_err[256] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+kvbfp_status cuda_fail(cudaError_t e, const char* what) {
+    snprintf(t_err, sizeof t_err, "%s: %s", what, cudaGetErrorString(e));
+    (void)cudaGetLastError();   // clear the sticky-less error state
+    return KVBFP_ERR_CUDA;
+}
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+kvbfp_status status_word(uint32_t** ptr) {
+    constexpr int kMaxDev = 64;
+    static uint32_t* cache[kMaxDev] = {nullptr};
+    int dev = 0;
+    KVBFP_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDev) return KVBFP_ERR_UNSUPPORTED;
+    if (!cache[dev]) {
+        uint32_t* p = nullptr;
+        KVBFP_CUDA(cudaGetSymbolAddress((void**)&p, g_status_word));
+        cache[dev] = p;
+    }
+    *ptr = cache[dev];
+    return KVBFP_OK;
+}
+
+}  // namespace kvbfp
+
+extern "C" {
+
+int32_t kvbfp_version(void) { return 100; }
+
+const char* kvbfp_status_string(kvbfp_status s) {
+    switch (s) {
+        case KVBFP_OK: return "ok";
+        case KVBFP_ERR_INVALID_ARG: return "invalid argument";
+        case KVBFP_ERR_UNSUPPORTED: return "unsupported format or shape";
+        case KVBFP_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+        case KVBFP_ERR_CAPACITY: return "cache capacity exceeded";
+        case KVBFP_ERR_WORKSPACE: return "workspace missing or too small";
+        case KVBFP_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+const char* kvbfp_last_cuda_error(void) { return kvbfp::t_err; }
+
+uint64_t kvbfp_launch_count(void) { return kvbfp::g_launches.load(std::memory_order_relaxed); }
+
+kvbfp_status kvbfp_plane_bytes(const kvbfp_format* fmt, size_t* mant_bytes, size_t* exp_bytes) {
+    kvbfp_status st = kvbfp::check_format(fmt);
+    if (st != KVBFP_OK) return st;
+    size_t rows = (size_t)fmt->batch * fmt->n_kv_heads * fmt->max_seq;
+    if (mant_bytes) *mant_bytes = rows * kvbfp::row_m_bytes(*fmt);
+    if (exp_bytes) *exp_bytes = rows * kvbfp::row_e_bytes(*fmt);
+    return KVBFP_OK;
+}
+
+kvbfp_status kvbfp_device_status(uint32_t* flags_out, void* stream) {
+    if (!flags_out) return KVBFP_ERR_INVALID_ARG;
+    uint32_t* w = nullptr;
+    kvbfp_status st = kvbfp::status_word(&w);
+    if (st != KVBFP_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    KVBFP_CUDA(cudaMemcpyAsync(flags_out, w, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
+    KVBFP_CUDA(cudaMemsetAsync(w, 0, sizeof(uint32_t), s));
+    KVBFP_CUDA(cudaStreamSynchronize(s));
+    return KVBFP_OK;
+}
+
+}  // extern "C"

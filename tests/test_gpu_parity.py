@@ -1,0 +1,339 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on the same seeded inputs.
+
+Bit-exact for permutations, exponent planes, mantissa planes, statistics and dequantised values;
+attention within 2e-3 of fp64 attention over the oracle's own cache, measured per (batch, query head)
+row as max_c |o_gpu - o_ref| / max_c |o_ref|.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from paper_2403_20137_b200 import binding as B
+from paper_2403_20137_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+ATTN_TOL = 2e-3
+P_GRID = [4, 6, 8]
+N_GRID = [16, 32, 64, 128]
+
+
+def dev(x):
+    return x.cuda().contiguous()
+
+
+def host(x):
+    return x.detach().cpu().numpy()
+
+
+def adversarial_rows(dtype, rows=96, seed=0):
+    """[1, rows, 2, 128] with the cases that break casts: exact .5 ties, clamp-zone values, zeros,
+    subnormals, +-max finite, a huge dynamic range between rows."""
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((1, rows, 2, 128)).astype(np.float32)
+    x *= np.exp2(rng.integers(-30, 30, size=(1, rows, 2, 1))).astype(np.float32)
+    x[0, 0] = 0.0                                             # all-zero rows
+    x[0, 1, :, :] = 0.0
+    x[0, 1, 0, 5] = 1.0                                       # a lone power of two
+    x[0, 2, 0, :] = np.arange(128) * 0.125 - 8.0              # dense dyadic grid: many exact ties
+    x[0, 2, 1, :] = np.arange(128) * 0.5 - 32.0
+    x[0, 3, 0, :] = np.float32(1e-40)                         # subnormal block
+    x[0, 3, 0, 7] = np.float32(3e-39)
+    x[0, 3, 1, :] = np.float32(3.0e38) * rng.choice([-1, 1], 128)   # near the largest finite value
+    x[0, 4, 0, :] = 1.0
+    x[0, 4, 0, ::16] = 1.96875                                # rounds up into the clamp zone (p=4: 7.875)
+    x[0, 4, 1, :] = -1.0
+    x[0, 4, 1, 1::16] = -1.9921875
+    x[0, 5, 0, :] = np.float32(2.0 ** -126)                   # smallest normal and below
+    x[0, 5, 0, 1::2] = np.float32(2.0 ** -127)
+    x[0, 5, 1, :] = np.float32(2.0 ** -149)
+    x[0, 6, :, :] = rng.integers(-7, 8, size=(2, 128)) * 0.25  # already on a coarse grid
+    t = torch.from_numpy(x)
+    return t.to(W.torch_dtype(dtype))
+
+
+def oracle_cache(oracle, k, v, dtype, block, p, max_seq, start=None, perm_k=None, perm_v=None):
+    Bn, T, H, d = k.shape
+    c = oracle.Cache(Bn, H, d, max_seq, block, p)
+    sp = np.zeros(Bn, dtype=np.int32) if start is None else np.asarray(start, dtype=np.int32)
+    oracle.append(c, W.to_oracle(k), None if v is None else W.to_oracle(v), dtype, sp, perm_k, perm_v)
+    return c
+
+
+def assert_planes_equal(gc, oc, lens, start=None):
+    """Compare the rows that were written; everything else is unspecified."""
+    Bn = gc.fmt.batch
+    for b in range(Bn):
+        s0 = 0 if start is None else int(start[b])
+        sl = slice(s0, s0 + int(lens[b]))
+        for name in ("k_mant", "k_exp", "v_mant", "v_exp"):
+            g = host(getattr(gc, name)[b, :, sl])
+            o = getattr(oc, name)[b, :, sl]
+            assert np.array_equal(g, o), f"{name} differs for batch {b}"
+
+
+# ------------------------------------------------------------------------------- append
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("p", P_GRID)
+@pytest.mark.parametrize("n", N_GRID)
+def test_append_bit_exact_format_grid(oracle, dtype, p, n):
+    k = adversarial_rows(dtype, seed=1)
+    v = adversarial_rows(dtype, seed=2)
+    rng = np.random.default_rng(3)
+    perm_k = np.stack([rng.permutation(128) for _ in range(2)]).astype(np.int32)
+    perm_v = np.stack([rng.permutation(128) for _ in range(2)]).astype(np.int32)
+    T = k.shape[1]
+    gc = B.Cache(1, 2, 128, 112, n, p, fill=0xA5)
+    start = torch.tensor([16], dtype=torch.int32)
+    B.append(gc, dev(k), dev(v), dev(start), dev(torch.from_numpy(perm_k)), dev(torch.from_numpy(perm_v)))
+    assert B.device_status() == 0
+    oc = oracle_cache(oracle, k, v, dtype, n, p, 112, start=[16], perm_k=perm_k, perm_v=perm_v)
+    assert_planes_equal(gc, oc, [T], start=[16])
+    # rows outside [16, 16+T) keep their fill
+    assert bool((gc.k_mant[0, :, :16] == 0xA5).all()) and bool((gc.k_exp[0, :, 16 + T:] == 0xA5).all())
+    # dequant parity (Eq. (1)), original channel order, both output types
+    for which, perm in (("k", perm_k), ("v", perm_v)):
+        for h in range(2):
+            ref = oracle.dequant(oc, which, 0, h, 16, T, perm=perm)
+            pd = dev(torch.from_numpy(perm))
+            got = host(B.dequant(gc, which, 0, h, 16, T, perm=pd))
+            assert np.array_equal(got.astype(np.float64), ref)
+            got16 = B.dequant(gc, which, 0, h, 16, T, perm=pd, out_dtype=torch.bfloat16)
+            assert np.array_equal(host(got16.float()).astype(np.float64), ref)
+    ref = oracle.dequant(oc, "k", 0, 1, 20, 7)
+    assert np.array_equal(host(B.dequant(gc, "k", 0, 1, 20, 7)).astype(np.float64), ref)
+
+
+def test_append_identity_and_single_plane(oracle):
+    w = W.CONFIGS[2]
+    k, v = W.make_kv(w, n_tokens=50)
+    gc = B.Cache(1, 32, 128, 64, 32, 4, fill=0)
+    B.append(gc, dev(k), None, dev(torch.zeros(1, dtype=torch.int32)))
+    oc = oracle_cache(oracle, k, None, "bf16", 32, 4, 64)
+    assert np.array_equal(host(gc.k_mant[0, :, :50]), oc.k_mant[0, :, :50])
+    assert np.array_equal(host(gc.k_exp[0, :, :50]), oc.k_exp[0, :, :50])
+    assert not bool(gc.v_mant.any())          # V untouched
+    B.append(gc, None, dev(v), dev(torch.zeros(1, dtype=torch.int32)))
+    oc2 = oracle_cache(oracle, v, None, "bf16", 32, 4, 64)
+    assert np.array_equal(host(gc.v_mant[0, :, :50]), oc2.k_mant[0, :, :50])
+
+
+def test_append_ragged_positions_and_flags(oracle):
+    """Per-sequence start positions; a sequence that would overflow is skipped whole and flagged."""
+    w = W.CONFIGS[3]
+    k, v = W.make_kv(w, n_tokens=3, batch=4)
+    gc = B.Cache(4, 32, 128, 32, 32, 4, fill=0x11)
+    start = [0, 29, 30, 7]
+    B.append(gc, dev(k), dev(v), dev(torch.tensor(start, dtype=torch.int32)))
+    assert B.device_status() == B.FLAG_POSITION
+    assert B.device_status() == 0                    # cleared by the read
+    assert bool((gc.k_mant[2] == 0x11).all()) and bool((gc.v_exp[2] == 0x11).all())
+    oc = oracle.Cache(4, 32, 128, 32, 32, 4)
+    ok = [0, 1, 3]
+    for b in ok:     # the oracle refuses an overflowing call, so feed it the sequences that fit
+        sub = oracle.Cache(1, 32, 128, 32, 32, 4)
+        oracle.append(sub, W.to_oracle(k[b:b + 1]), W.to_oracle(v[b:b + 1]), "bf16", np.array([start[b]], np.int32))
+        sl = slice(start[b], start[b] + 3)
+        assert np.array_equal(host(gc.k_mant[b, :, sl]), sub.k_mant[0, :, sl])
+        assert np.array_equal(host(gc.v_exp[b, :, sl]), sub.v_exp[0, :, sl])
+    del oc
+    bad = k.clone()
+    bad[0, 1, 3, 9] = float("inf")
+    B.append(gc, dev(bad), None, dev(torch.zeros(4, dtype=torch.int32)))
+    assert B.device_status() & B.FLAG_NONFINITE
+
+
+# ------------------------------------------------------------------------------- calibrate
+@pytest.mark.parametrize("cfg,T", [(1, 256), (2, 1000), (4, 777)])
+def test_calibrate_matches_oracle(oracle, cfg, T):
+    w = W.CONFIGS[cfg]
+    x = W.make_calibration(w, n_tokens=T)
+    st, perm, inv = B.calibrate(dev(x), w.n_kv_heads, 128)
+    assert B.device_status() == 0
+    st_o, perm_o, inv_o = oracle.calibrate(W.to_oracle(x), w.dtype, w.n_kv_heads, 128)
+    assert np.array_equal(host(st).astype(np.float64), st_o)
+    assert np.array_equal(host(perm), perm_o) and np.array_equal(host(inv), inv_o)
+
+
+def test_calibrate_ties_and_edge_cases(oracle):
+    """Duplicate statistics decide real outputs (bf16 magnitudes repeat): the order must be stable."""
+    rng = np.random.default_rng(4)
+    x = rng.integers(-3, 4, size=(40, 3, 128)).astype(np.float32)     # only 4 distinct magnitudes
+    xt = torch.from_numpy(x).to(torch.bfloat16)
+    st, perm, inv = B.calibrate(dev(xt), 3, 128)
+    st_o, perm_o, inv_o = oracle.calibrate(W.to_oracle(xt), "bf16", 3, 128)
+    assert np.array_equal(host(perm), perm_o) and np.array_equal(host(inv), inv_o)
+    # one token, and zero tokens (all statistics 0 -> identity order)
+    st, perm, _ = B.calibrate(dev(xt[:1]), 3, 128)
+    _, perm_o, _ = oracle.calibrate(W.to_oracle(xt[:1]), "bf16", 3, 128)
+    assert np.array_equal(host(perm), perm_o)
+    st, perm, _ = B.calibrate(dev(torch.zeros(1, 3, 128))[:0], 3, 128)
+    assert np.array_equal(host(perm), np.tile(np.arange(128, dtype=np.int32), (3, 1)))
+    assert not bool(st.any())
+
+
+def test_calibrate_l2_and_fold(oracle):
+    """Algorithm 1 verbatim: Euclidean row norms of W_k (given transposed), argsort, row gather."""
+    rng = np.random.default_rng(5)
+    H, d, d_in = 4, 128, 320
+    wk = rng.standard_normal((H * d, d_in)).astype(np.float32)
+    wk[rng.integers(0, H * d, size=20)] *= 15.0
+    x = torch.from_numpy(np.ascontiguousarray(wk.T))                  # [d_in, H, d]
+    st, perm, inv = B.calibrate(dev(x), H, d, stat=B.STAT_L2)
+    st_o, perm_o, inv_o = oracle.calibrate(x.numpy(), "f32", H, d, stat=oracle.STAT_L2)
+    assert np.allclose(host(st), st_o, rtol=1e-6, atol=0)
+    gp, go = host(perm), perm_o
+    for h in range(H):      # identical, or differing only between channels whose norms agree to 1e-12
+        for j in np.nonzero(gp[h] != go[h])[0]:
+            assert abs(st_o[h, gp[h, j]] - st_o[h, go[h, j]]) <= 1e-12 * st_o[h, go[h, j]]
+    folded = B.fold_perm(dev(torch.from_numpy(wk)), perm, H, d)
+    ref = oracle.fold_perm(wk.reshape(H, d, d_in).astype(np.float64), gp)
+    assert np.array_equal(host(folded).reshape(H, d, d_in).astype(np.float64), ref)
+    # Eq. (2): with both weights folded the products agree with the unfolded ones
+    wq = rng.standard_normal((H * d, d_in)).astype(np.float32)
+    fq = host(B.fold_perm(dev(torch.from_numpy(wq)), perm, H, d)).astype(np.float64)
+    fk = host(folded).astype(np.float64)
+    a = wq[:d].astype(np.float64).T @ wk[:d].astype(np.float64)
+    b = fq[:d].T @ fk[:d]
+    assert np.allclose(a, b, rtol=1e-12, atol=1e-12)
+
+
+# ------------------------------------------------------------------------------- decode attention
+def rel_err(got, ref):
+    """Per (batch, head) row: max |diff| / max |ref|."""
+    num = np.abs(got - ref).max(axis=-1)
+    den = np.abs(ref).max(axis=-1)
+    return float((num / np.maximum(den, 1e-30)).max())
+
+
+def run_decode_case(oracle, w, Bn, S, lens, block, p, impl, use_perm=True, perm_v=False, max_seq=None,
+                    chunk_tokens=0, q_mant_bits=0, scale=0.0, hint=0):
+    max_seq = max_seq or ((S + 15) // 16) * 16
+    k, v = W.make_kv(w, n_tokens=S, batch=Bn)
+    q = W.make_q(w, batch=Bn)
+    pk = pv = ipv = None
+    if use_perm:
+        _, pk, _ = oracle.calibrate(W.to_oracle(k.reshape(-1, w.n_kv_heads, 128)), w.dtype, w.n_kv_heads, 128)
+    if perm_v:
+        _, pv, ipv = oracle.calibrate(W.to_oracle(v.reshape(-1, w.n_kv_heads, 128)), w.dtype, w.n_kv_heads, 128)
+    oc = oracle_cache(oracle, k, v, w.dtype, block, p, max_seq, perm_k=pk, perm_v=pv)
+    ref = oracle.decode_attn(oc, W.to_oracle(q), w.dtype, w.n_q_heads, lens, perm_k=pk, inv_perm_v=ipv,
+                             softmax_scale=scale, q_mant_bits=q_mant_bits)
+    t = lambda a: None if a is None else dev(torch.from_numpy(a))
+    gc = B.Cache(Bn, w.n_kv_heads, 128, max_seq, block, p, fill=0xFF)    # unwritten rows: worst-case bytes
+    B.append(gc, dev(k), dev(v), dev(torch.zeros(Bn, dtype=torch.int32)), t(pk), t(pv))
+    out = B.decode_attn(gc, dev(q), dev(torch.tensor(lens, dtype=torch.int32)), perm_k=t(pk), inv_perm_v=t(ipv),
+                        softmax_scale=scale, impl=impl, chunk_tokens=chunk_tokens, q_mant_bits=q_mant_bits,
+                        max_len_hint=hint)
+    assert B.device_status() == 0
+    return host(out).astype(np.float64), ref
+
+
+IMPLS = [B.DECODE_SIMT, B.DECODE_MMA]
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_decode_config1(oracle, impl):
+    """Single head, fp32, block 16, 4-bit, four x20 outlier channels, 256 tokens."""
+    w = W.CONFIGS[1]
+    got, ref = run_decode_case(oracle, w, 1, 256, [256], 16, 4, impl)
+    assert rel_err(got, ref) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("p", P_GRID)
+@pytest.mark.parametrize("n", N_GRID)
+def test_decode_format_grid_ragged(oracle, impl, p, n):
+    """Llama-2-shaped heads, ragged lengths spanning several stages, tiles and a ragged tail."""
+    w = W.CONFIGS[2]
+    lens = [333, 1, 16, 200]
+    got, ref = run_decode_case(oracle, w, 4, 333, lens, n, p, impl, max_seq=400)
+    assert rel_err(got, ref) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_decode_gqa(oracle, impl):
+    w = W.CONFIGS[4]
+    lens = [700, 129]
+    got, ref = run_decode_case(oracle, w, 2, 700, lens, 32, 4, impl, perm_v=True)
+    assert rel_err(got, ref) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_decode_group_of_8_and_2(oracle, impl):
+    import dataclasses
+    for hq, hkv in ((16, 2), (4, 2)):
+        w = dataclasses.replace(W.CONFIGS[4], n_q_heads=hq, n_kv_heads=hkv)
+        got, ref = run_decode_case(oracle, w, 1, 150, [150], 32, 4, impl)
+        assert rel_err(got, ref) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_decode_empty_and_capacity_edges(oracle, impl):
+    w = W.CONFIGS[2]
+    got, ref = run_decode_case(oracle, w, 3, 128, [0, 128, 5], 32, 4, impl, max_seq=128)
+    assert not got[0].any() and not ref[0].any()          # empty sequence -> zeros
+    assert rel_err(got[1:], ref[1:]) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_decode_split_invariance(oracle, impl):
+    """The chunk count must not matter: 1, 2, 7 and 52 chunks agree with each other.  The fp32 kernel
+    agrees to 1e-5; the tensor-core kernel carries q and the softmax weights as two bf16 terms
+    (2^-16 relative each), and a different chunking moves the softmax reference point, so its runs
+    may differ from each other by a few 2^-16."""
+    w = W.CONFIGS[2]
+    S = 6600
+    outs = []
+    for chunk in (6656, 3328, 1024, 128):
+        got, ref = run_decode_case(oracle, w, 1, S, [S], 32, 4, impl, chunk_tokens=chunk)
+        assert rel_err(got, ref) <= ATTN_TOL
+        outs.append(got)
+    for o in outs[1:]:
+        assert rel_err(o, outs[0]) <= (1e-5 if impl == B.DECODE_SIMT else 1e-4)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_decode_bfp16_query_and_scale(oracle, impl):
+    w = W.CONFIGS[2]
+    got, ref = run_decode_case(oracle, w, 1, 300, [300], 32, 4, impl, q_mant_bits=8, scale=0.05)
+    assert rel_err(got, ref) <= ATTN_TOL
+    got, ref = run_decode_case(oracle, w, 1, 300, [300], 64, 4, impl, q_mant_bits=8)
+    assert rel_err(got, ref) <= ATTN_TOL
+
+
+def test_decode_len_hint_flag(oracle):
+    w = W.CONFIGS[2]
+    k, v = W.make_kv(w, n_tokens=256)
+    gc = B.Cache(1, 32, 128, 256, 32, 4)
+    z = dev(torch.zeros(1, dtype=torch.int32))
+    B.append(gc, dev(k), dev(v), z)
+    q = dev(W.make_q(w))
+    lens = dev(torch.tensor([256], dtype=torch.int32))
+    a = B.decode_attn(gc, q, lens, max_len_hint=128)
+    assert B.device_status() == B.FLAG_LEN_HINT
+    b = B.decode_attn(gc, q, dev(torch.tensor([128], dtype=torch.int32)))
+    assert B.device_status() == 0
+    assert torch.equal(a, b)                               # tokens past the hint were not read
+    B.decode_attn(gc, q, dev(torch.tensor([300], dtype=torch.int32)))
+    assert B.device_status() & B.FLAG_POSITION
+
+
+def test_ksort_improves_gpu_cache_quality(oracle):
+    """Direction of effect on the GPU path itself: K-sort lowers key MSE and score error."""
+    w = W.CONFIGS[2]
+    k, v = W.make_kv(w, n_tokens=512)
+    kd = dev(k)
+    _, perm, _ = B.calibrate(kd.reshape(-1, 32, 128), 32, 128)
+    z = dev(torch.zeros(1, dtype=torch.int32))
+    plain, sortd = B.Cache(1, 32, 128, 512, 32, 4), B.Cache(1, 32, 128, 512, 32, 4)
+    B.append(plain, kd, None, z)
+    B.append(sortd, kd, None, z, perm_k=perm)
+    mse_p = mse_s = 0.0
+    for h in range(32):
+        ref = k[0, :, h].float().cuda()
+        mse_p += float(((B.dequant(plain, "k", 0, h, 0, 512) - ref) ** 2).mean())
+        mse_s += float(((B.dequant(sortd, "k", 0, h, 0, 512, perm=perm) - ref) ** 2).mean())
+    assert mse_s < 0.85 * mse_p
