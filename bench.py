@@ -171,16 +171,27 @@ def run_reference(args, w, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, choices=[2, 3, 4])
     ap.add_argument("--decode-impl", default="auto", choices=["auto", "simt", "mma"])
     ap.add_argument("--ref-units", type=int, default=0, help="(batch, kv head) units per step of the reference arm (0 = sized for ~100 s)")
     ap.add_argument("--cpu-baseline-units", type=int, default=256)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=0, help="override the batch size (small cases for profiling)")
+    ap.add_argument("--seq", type=int, default=0, help="override the cached sequence length")
+    ap.add_argument("--mant-bits", type=int, default=0, choices=[0, 4, 6, 8])
+    ap.add_argument("--block", type=int, default=0, choices=[0, 16, 32, 64, 128])
+    ap.add_argument("--chunk", type=int, default=0, help="tokens per sequence chunk (0 = library default)")
+    ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
+    import dataclasses
+    over = {k: v for k, v in (("batch", args.batch), ("seq", args.seq), ("mant_bits", args.mant_bits),
+                              ("block", args.block)) if v}
+    if over:
+        w = dataclasses.replace(w, **over)
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -221,7 +232,8 @@ def main():
 
     def step():
         B.append(cache, k_new, v_new, start_pos, perm_k=perm_k)
-        B.decode_attn(cache, q, seq_lens, perm_k=perm_k, max_len_hint=S, impl=impl, out=out, workspace=ws)
+        B.decode_attn(cache, q, seq_lens, perm_k=perm_k, max_len_hint=S, impl=impl, out=out, workspace=ws,
+                      chunk_tokens=args.chunk)
 
     def barrier():
         if dist is not None:
@@ -263,18 +275,19 @@ def main():
         B.decode_step_host(cache, hk, hv, hq, start_pos, seq_lens, hout, staging, ws, perm_k=perm_k, max_len_hint=S,
                            impl=impl)
 
-    for _ in range(args.warmup):
+    n_e2e = 0 if args.no_e2e else args.steps
+    for _ in range(args.warmup if n_e2e else 0):
         step_host()
     barrier()
     f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     f0.record()
-    for _ in range(args.steps):
+    for _ in range(n_e2e):
         step_host()
     f1.record()
     barrier()
-    ms_e2e = f0.elapsed_time(f1)
+    ms_e2e = f0.elapsed_time(f1) if n_e2e else float("nan")
     clocks = sampler.stop() if rank == 0 else None
-    e2e_ok = bool(torch.allclose(hout.to(dev), out, rtol=0, atol=0))
+    e2e_ok = bool(torch.equal(hout.to(dev), out)) if n_e2e else None
 
     # ---- max over ranks -----------------------------------------------------------------------------
     if dist is not None:

@@ -61,8 +61,8 @@ def lib():
     """Load (building in-tree if the sources are newer) the CUDA library; raises if impossible."""
     global _lib
     if _lib is None:
-        path = _build.LIB
-        if not os.path.exists(path) or os.environ.get("KVBFP_REBUILD"):
+        path = os.environ.get("KVBFP_LIB") or _build.LIB      # KVBFP_LIB: another build of the same library
+        if path == _build.LIB and (not os.path.exists(path) or os.environ.get("KVBFP_REBUILD")):
             path = _build.build()
         L = C.CDLL(path)
         L.kvbfp_version.restype = C.c_int32

@@ -23,13 +23,13 @@ def _deps_mtime():
     return max(os.path.getmtime(f) for f in files)
 
 
-def _compile(src):
-    obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+def _compile(src, obj_dir=None, extra=()):
+    obj = os.path.join(obj_dir or OBJ_DIR, os.path.basename(src)[:-3] + ".o")
     hdr_time = max(os.path.getmtime(os.path.join(CSRC, f)) for f in os.listdir(CSRC) if f.endswith(".cuh"))
     hdr_time = max(hdr_time, os.path.getmtime(os.path.join(INCLUDE, "kvbfp.h")), os.path.getmtime(__file__))
     if os.path.exists(obj) and os.path.getmtime(obj) >= max(os.path.getmtime(src), hdr_time):
         return obj, ""
-    r = subprocess.run(["nvcc", *NVCC_FLAGS, "-c", src, "-o", obj], capture_output=True, text=True)
+    r = subprocess.run(["nvcc", *NVCC_FLAGS, *extra, "-c", src, "-o", obj], capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}\n{r.stderr}")
     return obj, r.stderr
@@ -53,6 +53,18 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
     return LIB
+
+
+def build_variant(out, defines, obj_dir):
+    """Development aid: the same sources with extra -D flags into another .so (tuning sweeps)."""
+    os.makedirs(obj_dir, exist_ok=True)
+    extra = tuple("-D" + d for d in defines)
+    with ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as ex:
+        results = list(ex.map(lambda src: _compile(src, obj_dir, extra), sources()))
+    objs = [o for o, _ in results]
+    subprocess.run(["nvcc", "-shared", "-o", out, *objs, "-gencode", "arch=compute_100a,code=sm_100a", "-lcudart"],
+                   check=True)
+    return out
 
 
 if __name__ == "__main__":

@@ -132,6 +132,7 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
     a.n_chunks = (a.len_cap + chunk - 1) / chunk;
     st = status_word(&a.status);
     if (st != KVBFP_OK) return st;
+    a.mulhi4 = 1u << 28; a.mulhi8 = 1u << 24; a.mulhi12 = 1u << 20;
 
     cudaStream_t s = (cudaStream_t)stream;
     st = (impl == KVBFP_DECODE_SIMT) ? launch_decode_simt(a, s) : launch_decode_mma(a, s);

@@ -27,6 +27,9 @@ struct DecodeArgs {
     int n_chunks;
     int len_cap;              // min(max_len_hint, max_seq)
     uint32_t* status;
+    // 2^(32-k): multiplying by these and keeping the high word is a right shift by k that runs on the
+    // multiply-add pipe instead of the integer pipe (passed at run time so that it stays a multiply)
+    uint32_t mulhi4, mulhi8, mulhi12;
 };
 
 kvbfp_status launch_decode_simt(const DecodeArgs& a, cudaStream_t s);

@@ -15,6 +15,10 @@
 // where the 8 columns are four query heads times (hi, lo) bf16 halves of q, so q keeps ~16 bits.
 // Output: O^T[16 slots x 8 cols] += V^T[16 slots x 16 tokens] . P^T[16 tokens x 8 cols], with the
 // softmax weights split into hi/lo halves the same way.  Accumulators are fp32.
+//
+// The integer pipe (logic ops, shifts, byte permutes) is what limits this kernel, so half of the
+// shifts are issued as multiply-high on the multiply-add pipe and block weights come from a
+// 256-entry table in shared memory instead of being rebuilt from the exponent byte.
 #include <math.h>
 
 #include "decode.cuh"
@@ -22,10 +26,32 @@
 namespace kvbfp {
 namespace {
 
-constexpr int kWarps = 4;
-constexpr int kMT = 2;                 // 16-token MMA row tiles per stage
+// Tuning knobs (compile-time; the defaults are the measured best on B200).
+#ifndef KVBFP_WARPS
+#define KVBFP_WARPS 4
+#endif
+#ifndef KVBFP_MT
+#define KVBFP_MT 2
+#endif
+#ifndef KVBFP_STAGES
+#define KVBFP_STAGES 3
+#endif
+#ifndef KVBFP_SHIFT_MULHI
+#define KVBFP_SHIFT_MULHI 0            // 1: shifts by 4 and 12 as multiply-high on the multiply-add pipe (slower on B200)
+#endif
+#ifndef KVBFP_MIN_CTAS
+#define KVBFP_MIN_CTAS 1               // resident thread blocks per SM the register allocation must allow
+#endif
+#ifndef KVBFP_QF_SMEM
+#define KVBFP_QF_SMEM 0                // 1: keep the query fragments in shared memory instead of registers
+#endif
+#ifndef KVBFP_K_ACC_SPLIT
+#define KVBFP_K_ACC_SPLIT 1            // 1: two independent accumulator chains for the score MMAs
+#endif
+
+constexpr int kWarps = KVBFP_WARPS;
+constexpr int kMT = KVBFP_MT;          // 16-token MMA row tiles per stage
 constexpr int kTile = 16 * kMT;        // tokens per stage
-constexpr uint32_t kWaitSpins = 1u << 20;
 
 // ------------------------------------------------------------------ PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -36,20 +62,29 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+// Bounded wait on a phase of an mbarrier.  Each try suspends the warp in hardware for up to
+// kWaitHintNs before it reports "not yet", so a waiting warp does not burn issue slots; after
+// kWaitTries tries the wait gives up and reports failure instead of spinning for ever.
+constexpr uint32_t kWaitHintNs = 1000000u;
+constexpr uint32_t kWaitTries = 2000u;
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .u32 n;\n\t"
+        "mov.u32 n, 0;\n\t"
+        "KVBFP_WAIT:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "@p bra KVBFP_DONE;\n\t"
+        "add.u32 n, n, 1;\n\t"
+        "setp.lt.u32 q, n, %4;\n\t"
+        "@q bra KVBFP_WAIT;\n\t"
+        "KVBFP_DONE:\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kWaitHintNs), "r"(kWaitTries) : "memory");
     return ok != 0;
-}
-// Bounded wait: gives up after kWaitSpins polls instead of spinning for ever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-    for (uint32_t i = 0; i < kWaitSpins; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -57,7 +92,7 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
@@ -76,6 +111,23 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
     asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
     return d;
 }
+// One three-input logic instruction; LUT is the truth table (0x6A = (a & b) ^ c, 0xEA = (a & b) | c).
+template <int LUT>
+__device__ __forceinline__ uint32_t lop3(uint32_t a, uint32_t b, uint32_t c) {
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, %4;" : "=r"(d) : "r"(a), "r"(b), "r"(c), "n"(LUT));
+    return d;
+}
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
 
 // bf16 bit pattern of 2^(e8 - 127 - (P-2)); subnormal results down to 2^-133 are exact.
 template <int P>
@@ -85,7 +137,7 @@ __device__ __forceinline__ uint32_t weight_bf16(uint32_t e8) {
 }
 
 // Format constants of the "or under 128.0" conversion.  The field with its sign bit flipped is
-// M + 2^(P-1) (P = 4, 6); the value built is 128 + 2^(P-1) + M, so the bias to remove is kBias.
+// M + 2^(P-1) (P = 4, 6); the value built is 128 + 2^(P-1) + M, so the bias to remove is `bias`.
 template <int P> struct Fmt;
 template <> struct Fmt<4> { static constexpr uint32_t mask = 0x000F000Fu, magic = 0x43084308u, bias = 0xC308C308u; };  // -136
 template <> struct Fmt<6> { static constexpr uint32_t mask = 0x003F003Fu, magic = 0x43204320u, bias = 0xC320C320u; };  // -160
@@ -98,10 +150,10 @@ struct Wgt {
     uint32_t s16;   // 16 * s   (8-bit mantissas only)
 };
 template <int P>
-__device__ __forceinline__ Wgt make_wgt(uint32_t s2) {
+__device__ __forceinline__ Wgt make_wgt(uint32_t s2, uint32_t c2) {
     Wgt w;
     w.s = s2;
-    w.c = mul_bf16x2(s2, Fmt<P>::bias);
+    w.c = c2;
     w.s16 = (P == 8) ? mul_bf16x2(s2, 0x41804180u) : 0u;   // 16.0
     return w;
 }
@@ -111,13 +163,29 @@ template <int P>
 __device__ __forceinline__ uint32_t cvt_pair(uint32_t x, const Wgt& w) {
     if (P == 8) {
         // byte = 16*H + L, H signed high nibble, L unsigned low nibble
-        uint32_t lo = (x & 0x000F000Fu) | 0x43004300u;                 // 128 + L
-        uint32_t hi = ((x >> 4) & 0x000F000Fu) ^ 0x43084308u;          // 136 + H
+        uint32_t lo = lop3<0xEA>(x, 0x000F000Fu, 0x43004300u);         // (x & m) | 128.0  = 128 + L
+        uint32_t hi = lop3<0x6A>(x >> 4, 0x000F000Fu, 0x43084308u);    // (x & m) ^ 136.0  = 136 + H
         uint32_t v = fma_bf16x2(hi, w.s16, w.c);                       // (16H - 128) * 2^e, exact
         return fma_bf16x2(lo, w.s, v);                                 // (16H + L) * 2^e, exact
     }
-    return fma_bf16x2((x & Fmt<P>::mask) ^ Fmt<P>::magic, w.s, w.c);
+    return fma_bf16x2(lop3<0x6A>(x, Fmt<P>::mask, Fmt<P>::magic), w.s, w.c);   // (x & mask) ^ magic in one op
 }
+
+// Right shifts of a packed word by 4, 8 and 12; two of the three run on the multiply-add pipe.
+struct Shifts {
+    uint32_t m4, m12;
+    __device__ __forceinline__ void apply(uint32_t x, uint32_t& x4, uint32_t& x8, uint32_t& x12) const {
+#if KVBFP_SHIFT_MULHI
+        x4 = __umulhi(x, m4);
+        x8 = x >> 8;
+        x12 = __umulhi(x, m12);
+#else
+        x4 = x >> 4;
+        x8 = x >> 8;
+        x12 = x >> 12;
+#endif
+    }
+};
 
 // Slot (within the 128-slot row) that the K-side unpack puts at k-position kk of k-step ks for lane
 // column t; kk = 0..3 stands for k = 2t, 2t+1, 2t+8, 2t+9 of the m16n8k16 fragment.
@@ -128,53 +196,64 @@ __host__ __device__ __forceinline__ int k_slot(int ks, int t, int kk) {
     return 32 * t + 4 * ks + kk;
 }
 
-// Two A registers (k = 2t..2t+1 and k = 2t+8..2t+9) of k-step ks from a lane's 32-slot chunk w[P].
+// Two A registers (k = 2t..2t+1 and k = 2t+8..2t+9) of k-steps ks and ks+1 (ks even) from a lane's
+// 32-slot chunk w[P].
 template <int P>
-__device__ __forceinline__ void k_pairs(const uint32_t (&w)[P], int ks, const Wgt& wg, uint32_t& r0, uint32_t& r1) {
+__device__ __forceinline__ void k_pairs2(const uint32_t (&w)[P], int ks, const Wgt& wg, const Shifts& sh,
+                                         uint32_t (&r)[4]) {
     if (P == 4) {
-        const uint32_t x = w[ks >> 1] >> (8 * (ks & 1));
-        r0 = cvt_pair<4>(x, wg);
-        r1 = cvt_pair<4>(x >> 4, wg);
+        uint32_t x4, x8, x12;
+        sh.apply(w[ks >> 1], x4, x8, x12);
+        r[0] = cvt_pair<4>(w[ks >> 1], wg);
+        r[1] = cvt_pair<4>(x4, wg);
+        r[2] = cvt_pair<4>(x8, wg);
+        r[3] = cvt_pair<4>(x12, wg);
     } else if (P == 8) {
-        r0 = cvt_pair<8>(w[ks], wg);
-        r1 = cvt_pair<8>(w[ks] >> 8, wg);
+        r[0] = cvt_pair<8>(w[ks], wg);
+        r[1] = cvt_pair<8>(w[ks] >> 8, wg);
+        r[2] = cvt_pair<8>(w[ks + 1], wg);
+        r[3] = cvt_pair<8>(w[ks + 1] >> 8, wg);
     } else {
-        uint32_t f[4];
+        uint32_t f[8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int bit = 6 * (4 * ks + j), word = bit >> 5, sh = bit & 31;
-            f[j] = (sh + 6 > 32) ? __funnelshift_r(w[word], w[(word + 1) % P], sh) : (w[word] >> sh);
+        for (int j = 0; j < 8; ++j) {
+            const int bit = 6 * (4 * ks + j), word = bit >> 5, s = bit & 31;
+            f[j] = (s + 6 > 32) ? __funnelshift_r(w[word], w[(word + 1) % P], s) : (w[word] >> s);
         }
-        r0 = cvt_pair<6>(prmt(f[0], f[1], 0x5410u), wg);
-        r1 = cvt_pair<6>(prmt(f[2], f[3], 0x5410u), wg);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) r[j] = cvt_pair<6>(prmt(f[2 * j], f[2 * j + 1], 0x5410u), wg);
     }
 }
 
-// V side: registers (slot 2r, token pair) and (slot 2r+1, token pair) from the two tokens' 16-slot
-// pieces wa[P/2*... ] (P/2 words each).
+// V side: registers for MMA row pairs r and r+1 (r even): (slot 2r, 2r+1, 2r+2, 2r+3) x (token pair),
+// from the two tokens' 16-slot pieces wa, wb (P/2 words each).
 template <int P>
-__device__ __forceinline__ void v_pairs(const uint32_t* wa, const uint32_t* wb, int r, const Wgt& wg, uint32_t& r0,
-                                        uint32_t& r1) {
+__device__ __forceinline__ void v_pairs2(const uint32_t* wa, const uint32_t* wb, int r, const Wgt& wg, const Shifts& sh,
+                                         uint32_t (&o)[4]) {
     if (P == 4) {
-        // word i = slots 8i..8i+7; halfword h of word i = slots 8i+4h..; slot 2r -> i = r>>2, h = (r>>1)&1, nibble 2(r&1)
-        const uint32_t x = prmt(wa[r >> 2], wb[r >> 2], ((r >> 1) & 1) ? 0x7632u : 0x5410u) >> (8 * (r & 1));
-        r0 = cvt_pair<4>(x, wg);
-        r1 = cvt_pair<4>(x >> 4, wg);
+        // word i = slots 8i..8i+7; halfword h of word i = slots 8i+4h..8i+4h+3 = rows 2r..2r+3 with r = 4i+2h
+        const uint32_t x = prmt(wa[r >> 2], wb[r >> 2], ((r >> 1) & 1) ? 0x7632u : 0x5410u);
+        uint32_t x4, x8, x12;
+        sh.apply(x, x4, x8, x12);
+        o[0] = cvt_pair<4>(x, wg);
+        o[1] = cvt_pair<4>(x4, wg);
+        o[2] = cvt_pair<4>(x8, wg);
+        o[3] = cvt_pair<4>(x12, wg);
     } else if (P == 8) {
-        // word i = slots 4i..4i+3; slots 2r, 2r+1 = halfword (r&1) of word r>>1
-        const uint32_t x = prmt(wa[r >> 1], wb[r >> 1], (r & 1) ? 0x7632u : 0x5410u);
-        r0 = cvt_pair<8>(x, wg);
-        r1 = cvt_pair<8>(x >> 8, wg);
+        // word i = slots 4i..4i+3; slots 2r..2r+3 = word r>>1
+        const uint32_t xl = prmt(wa[r >> 1], wb[r >> 1], 0x5410u), xh = prmt(wa[r >> 1], wb[r >> 1], 0x7632u);
+        o[0] = cvt_pair<8>(xl, wg);
+        o[1] = cvt_pair<8>(xl >> 8, wg);
+        o[2] = cvt_pair<8>(xh, wg);
+        o[3] = cvt_pair<8>(xh >> 8, wg);
     } else {
-        uint32_t fa[2], fb[2];
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int bit = 6 * (2 * r + j), word = bit >> 5, sh = bit & 31;
-            fa[j] = (sh + 6 > 32) ? __funnelshift_r(wa[word], wa[(word + 1) % 3], sh) : (wa[word] >> sh);
-            fb[j] = (sh + 6 > 32) ? __funnelshift_r(wb[word], wb[(word + 1) % 3], sh) : (wb[word] >> sh);
+        for (int j = 0; j < 4; ++j) {
+            const int bit = 6 * (2 * r + j), word = bit >> 5, s = bit & 31;
+            const uint32_t fa = (s + 6 > 32) ? __funnelshift_r(wa[word], wa[(word + 1) % 3], s) : (wa[word] >> s);
+            const uint32_t fb = (s + 6 > 32) ? __funnelshift_r(wb[word], wb[(word + 1) % 3], s) : (wb[word] >> s);
+            o[j] = cvt_pair<6>(prmt(fa, fb, 0x5410u), wg);
         }
-        r0 = cvt_pair<6>(prmt(fa[0], fb[0], 0x5410u), wg);
-        r1 = cvt_pair<6>(prmt(fa[1], fb[1], 0x5410u), wg);
     }
 }
 
@@ -247,22 +326,34 @@ template <int P, int N>
 struct Geo {
     static constexpr int D = kHeadDim;
     static constexpr int ROW_M = D * P / 8, ROW_E = D / N;
-    static constexpr int STAGES = (P == 4) ? 4 : 3;
+    static constexpr int STAGES = KVBFP_STAGES;
     static constexpr int KM_OFF = 0;
     static constexpr int VM_OFF = kTile * ROW_M;
     static constexpr int KE_OFF = 2 * kTile * ROW_M;
     static constexpr int VE_OFF = KE_OFF + kTile * ROW_E;
     static constexpr int STAGE_BYTES = 2 * kTile * (ROW_M + ROW_E);
     static constexpr int WARP_BYTES = STAGES * STAGE_BYTES;
-    static constexpr int SMEM_BYTES = kWarps * WARP_BYTES + kWarps * STAGES * 8;
+    static constexpr int LUT_OFF = kWarps * WARP_BYTES;                 // uint2[256]
+    static constexpr int BAR_OFF = LUT_OFF + 256 * 8;
+    static constexpr int QF_OFF = BAR_OFF + kWarps * STAGES * 8;        // uint2[NT][8][32] per warp (optional)
+    static constexpr int QF_WARP_BYTES = 8 * 32 * 8;                    // per n-tile
+    template <int NT> static constexpr int smem_bytes() { return QF_OFF + (KVBFP_QF_SMEM ? kWarps * NT * QF_WARP_BYTES : 0); }
 };
 
 template <int P, int N, int NT>
-__global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
+__global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(DecodeArgs a) {
     using G_ = Geo<P, N>;
     constexpr int D = kHeadDim, ROW_M = G_::ROW_M, ROW_E = G_::ROW_E, STAGES = G_::STAGES;
     constexpr int NBK = (N == 16) ? 2 : 1;            // blocks inside a K lane chunk of 32 slots
     extern __shared__ __align__(128) uint8_t smem[];
+
+    // weight table: entry e = (2^(e-127-(P-2)) twice as bf16x2, the same times the negated bias)
+    uint2* lut = reinterpret_cast<uint2*>(smem + G_::LUT_OFF);
+    for (int e = threadIdx.x; e < 256; e += kWarps * 32) {
+        const uint32_t s2 = weight_bf16<P>((uint32_t)e) * 0x00010001u;
+        lut[e] = make_uint2(s2, mul_bf16x2(s2, Fmt<P>::bias));
+    }
+    __syncthreads();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
@@ -289,7 +380,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
 
     uint8_t* wsm = smem + warp * G_::WARP_BYTES;
     const uint32_t wsm_u32 = smem_u32(wsm);
-    const uint32_t bar0 = smem_u32(smem + kWarps * G_::WARP_BYTES + warp * STAGES * 8);
+    const uint32_t bar0 = smem_u32(smem + G_::BAR_OFF + warp * STAGES * 8);
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < STAGES; ++s) mbar_init(bar0 + 8 * s, 1);
@@ -298,25 +389,31 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
     }
     __syncwarp();
 
-    const int64_t row0 = ((int64_t)b * Hkv + hk) * a.fmt.max_seq;
+    const int64_t row0 = ((int64_t)b * Hkv + hk) * a.fmt.max_seq + t0;
+    const uint8_t* gkm = a.k_mant + row0 * ROW_M;
+    const uint8_t* gvm = a.v_mant + row0 * ROW_M;
+    const uint8_t* gke = a.k_exp + row0 * ROW_E;
+    const uint8_t* gve = a.v_exp + row0 * ROW_E;
+    const int n_tok = t1 - t0;
     auto issue = [&](int stage, int tile) {      // lane 0 only
-        const int tb = t0 + tile * kTile;
-        int rows = t1 - tb;
+        const int off = tile * kTile;
+        int rows = n_tok - off;
         rows = rows >= kTile ? kTile : ((rows + 15) & ~15);     // whole 16-token groups; stays below max_seq
         const uint32_t bar = bar0 + 8 * stage;
         const uint32_t dst = wsm_u32 + stage * G_::STAGE_BYTES;
         mbar_expect_tx(bar, (uint32_t)(2 * rows * (ROW_M + ROW_E)));
-        bulk_g2s(dst + G_::KM_OFF, a.k_mant + (row0 + tb) * ROW_M, rows * ROW_M, bar);
-        bulk_g2s(dst + G_::VM_OFF, a.v_mant + (row0 + tb) * ROW_M, rows * ROW_M, bar);
-        bulk_g2s(dst + G_::KE_OFF, a.k_exp + (row0 + tb) * ROW_E, rows * ROW_E, bar);
-        bulk_g2s(dst + G_::VE_OFF, a.v_exp + (row0 + tb) * ROW_E, rows * ROW_E, bar);
+        bulk_g2s(dst + G_::KM_OFF, gkm + off * ROW_M, rows * ROW_M, bar);
+        bulk_g2s(dst + G_::VM_OFF, gvm + off * ROW_M, rows * ROW_M, bar);
+        bulk_g2s(dst + G_::KE_OFF, gke + off * ROW_E, rows * ROW_E, bar);
+        bulk_g2s(dst + G_::VE_OFF, gve + off * ROW_E, rows * ROW_E, bar);
     };
     if (lane == 0) {
         for (int s = 0; s < STAGES && s < n_tiles; ++s) issue(s, s);
     }
 
-    // B fragments of pi(q): 16 registers per n-tile
-    uint32_t qf[NT][8][2];
+    // B fragments of pi(q): 16 registers per n-tile, or a per-warp copy in shared memory
+#if KVBFP_QF_SMEM
+    uint2* qsm = reinterpret_cast<uint2*>(smem + G_::QF_OFF + warp * NT * G_::QF_WARP_BYTES) + lane;
     {
         const uint4* src = reinterpret_cast<const uint4*>(a.qfrag) + (((int64_t)b * Hkv + hk) * NT) * (4 * 32);
 #pragma unroll
@@ -324,9 +421,28 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const uint4 v = __ldg(src + (nt * 4 + j) * 32 + lane);
-                qf[nt][2 * j][0] = v.x; qf[nt][2 * j][1] = v.y; qf[nt][2 * j + 1][0] = v.z; qf[nt][2 * j + 1][1] = v.w;
+                qsm[(nt * 8 + 2 * j) * 32] = make_uint2(v.x, v.y);
+                qsm[(nt * 8 + 2 * j + 1) * 32] = make_uint2(v.z, v.w);
             }
     }
+    __syncwarp();
+#define QF(nt, ks) (qsm[((nt) * 8 + (ks)) * 32])
+#else
+    uint2 qf[NT][8];
+    {
+        const uint4* src = reinterpret_cast<const uint4*>(a.qfrag) + (((int64_t)b * Hkv + hk) * NT) * (4 * 32);
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint4 v = __ldg(src + (nt * 4 + j) * 32 + lane);
+                qf[nt][2 * j] = make_uint2(v.x, v.y);
+                qf[nt][2 * j + 1] = make_uint2(v.z, v.w);
+            }
+    }
+#define QF(nt, ks) (qf[nt][ks])
+#endif
+    const Shifts sh{a.mulhi4, a.mulhi12};
 
     float o[NT][8][4];
 #pragma unroll
@@ -339,14 +455,22 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) { m_run[nt] = -INFINITY; l_run[nt] = 0.f; }
 
+    // per-lane byte offsets inside a stage
+    const int k_off = G_::KM_OFF + g * ROW_M + t * (4 * P);                       // + mt*16*ROW_M, + 8*ROW_M
+    const int ke_off = G_::KE_OFF + g * ROW_E + ((N == 16) ? 2 * t : (N == 32) ? t : (N == 64) ? (t >> 1) : 0);
+    const int v_off = G_::VM_OFF + t * ROW_M + g * (2 * P);                       // + (mt*16 + 4k)*ROW_M
+    const int ve_off = G_::VE_OFF + t * ROW_E + (16 * g) / N;
+    const int src_lo = 4 * t + (g >> 1), src_hi = 4 * (t + 4) + (g >> 1);
+    const bool odd_col = (g & 1) != 0;
+
     bool timed_out = false;
     for (int it = 0; it < n_tiles; ++it) {
         const int stage = it % STAGES;
         const uint32_t parity = (uint32_t)(it / STAGES) & 1u;
         if (!mbar_wait_bounded(bar0 + 8 * stage, parity)) { timed_out = true; break; }
         const uint8_t* st = wsm + stage * G_::STAGE_BYTES;
-        const int tb = t0 + it * kTile;
-        const int n_live = t1 - tb;                   // tokens of this tile that exist (may exceed kTile)
+        const int n_live = n_tok - it * kTile;        // tokens of this tile that exist (may exceed kTile)
+        const bool full = n_live >= kTile;
 
         // ---- scores -------------------------------------------------------------
         float sc[kMT][NT][2];
@@ -357,11 +481,10 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
                 for (int nt = 0; nt < NT; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = -INFINITY;
                 continue;
             }
-            const int ra = mt * 16 + g, rb = ra + 8;
             uint32_t wa[P], wb[P];
             {
-                const uint8_t* pa = st + G_::KM_OFF + ra * ROW_M + t * (4 * P);
-                const uint8_t* pb = st + G_::KM_OFF + rb * ROW_M + t * (4 * P);
+                const uint8_t* pa = st + k_off + mt * 16 * ROW_M;
+                const uint8_t* pb = pa + 8 * ROW_M;
                 if (P == 6) {
 #pragma unroll
                     for (int i = 0; i < 3; ++i) {
@@ -378,34 +501,48 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
                 }
             }
             Wgt ga[NBK], gb[NBK];
-            {
-                const int eb = (N == 16) ? 2 * t : (N == 32) ? t : (N == 64) ? (t >> 1) : 0;
 #pragma unroll
-                for (int k = 0; k < NBK; ++k) {
-                    const uint32_t sa = weight_bf16<P>(st[G_::KE_OFF + ra * ROW_E + eb + k]);
-                    const uint32_t sb = weight_bf16<P>(st[G_::KE_OFF + rb * ROW_E + eb + k]);
-                    ga[k] = make_wgt<P>(sa * 0x00010001u);
-                    gb[k] = make_wgt<P>(sb * 0x00010001u);
-                }
+            for (int k = 0; k < NBK; ++k) {
+                const uint2 la = lut[st[ke_off + mt * 16 * ROW_E + k]];
+                const uint2 lb = lut[st[ke_off + (mt * 16 + 8) * ROW_E + k]];
+                ga[k] = make_wgt<P>(la.x, la.y);
+                gb[k] = make_wgt<P>(lb.x, lb.y);
             }
-            float acc[NT][4];
+            constexpr int NACC = KVBFP_K_ACC_SPLIT ? 2 : 1;
+            float acc[NT][NACC][4];
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt) acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+            for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
+                for (int c = 0; c < NACC; ++c) acc[nt][c][0] = acc[nt][c][1] = acc[nt][c][2] = acc[nt][c][3] = 0.f;
+#pragma unroll
+            for (int ks = 0; ks < 8; ks += 2) {
                 const int kb = (NBK == 2) ? (ks >> 2) : 0;
-                uint32_t a0, a1, a2, a3;
-                k_pairs<P>(wa, ks, ga[kb], a0, a2);
-                k_pairs<P>(wb, ks, gb[kb], a1, a3);
+                uint32_t ra[4], rb[4];
+                k_pairs2<P>(wa, ks, ga[kb], sh, ra);
+                k_pairs2<P>(wb, ks, gb[kb], sh, rb);
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma_bf16(acc[nt], a0, a1, a2, a3, qf[nt][ks][0], qf[nt][ks][1]);
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint2 q0 = QF(nt, ks), q1 = QF(nt, ks + 1);
+                    mma_bf16(acc[nt][0], ra[0], rb[0], ra[1], rb[1], q0.x, q0.y);
+                    mma_bf16(acc[nt][NACC - 1], ra[2], rb[2], ra[3], rb[3], q1.x, q1.y);
+                }
             }
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                const float s0 = (acc[nt][0] + acc[nt][1]) * a.scale_log2e;
-                const float s1 = (acc[nt][2] + acc[nt][3]) * a.scale_log2e;
-                sc[mt][nt][0] = (ra < n_live) ? s0 : -INFINITY;     // select, not arithmetic: rows past the
-                sc[mt][nt][1] = (rb < n_live) ? s1 : -INFINITY;     // end may hold anything
+                float s0 = acc[nt][0][0] + acc[nt][0][1], s1 = acc[nt][0][2] + acc[nt][0][3];
+                if (NACC == 2) {
+                    s0 += acc[nt][1][0] + acc[nt][1][1];
+                    s1 += acc[nt][1][2] + acc[nt][1][3];
+                }
+                sc[mt][nt][0] = s0 * a.scale_log2e;
+                sc[mt][nt][1] = s1 * a.scale_log2e;
+            }
+            if (!full) {       // select, not arithmetic: rows past the end may hold anything
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    if (mt * 16 + g >= n_live) sc[mt][nt][0] = -INFINITY;
+                    if (mt * 16 + g + 8 >= n_live) sc[mt][nt][1] = -INFINITY;
+                }
             }
         }
 
@@ -427,7 +564,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const float m_new = fmaxf(m_run[nt], tmax[nt]);
-                const float alpha = (m_run[nt] == -INFINITY) ? 0.f : exp2f(m_run[nt] - m_new);
+                const float alpha = (m_run[nt] == -INFINITY) ? 0.f : ex2_approx(m_run[nt] - m_new);
                 m_run[nt] = m_new;
                 l_run[nt] *= alpha;
 #pragma unroll
@@ -441,36 +578,34 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
 #pragma unroll
         for (int mt = 0; mt < kMT; ++mt) {
             if (mt * 16 >= n_live) continue;
-            // softmax weights of this lane's tokens (g and g+8) for its query column pair
+            // softmax weights of this lane's tokens (g and g+8), then the B fragment of P^T for lane (g, t):
+            // column g = (query g/2, half g%2); tokens t, t+4 | t+8, t+12
             uint32_t pb[NT][2];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                const float p0 = (m_run[nt] == -INFINITY) ? 0.f : exp2f(sc[mt][nt][0] - m_run[nt]);
-                const float p1 = (m_run[nt] == -INFINITY) ? 0.f : exp2f(sc[mt][nt][1] - m_run[nt]);
+                const float p0 = ex2_approx(sc[mt][nt][0] - m_run[nt]);
+                const float p1 = ex2_approx(sc[mt][nt][1] - m_run[nt]);
                 l_run[nt] += p0 + p1;
-                // B fragment of P^T for lane (g, t): column g = (query g/2, half g%2); tokens t, t+4, t+8, t+12
-                const int src_lo = 4 * t + (g >> 1), src_hi = 4 * (t + 4) + (g >> 1);
                 const float v0 = __shfl_sync(0xffffffffu, p0, src_lo);   // token t
                 const float v1 = __shfl_sync(0xffffffffu, p0, src_hi);   // token t+4
                 const float v2 = __shfl_sync(0xffffffffu, p1, src_lo);   // token t+8
                 const float v3 = __shfl_sync(0xffffffffu, p1, src_hi);   // token t+12
-                float v[4] = {v0, v1, v2, v3};
-                uint32_t h[4];
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const __nv_bfloat16 hi = __float2bfloat16_rn(v[k]);
-                    const __nv_bfloat16 lo = __float2bfloat16_rn(v[k] - __bfloat162float(hi));
-                    h[k] = __bfloat16_as_ushort((g & 1) ? lo : hi);
-                }
-                pb[nt][0] = h[0] | (h[1] << 16);
-                pb[nt][1] = h[2] | (h[3] << 16);
+                // hi half = the value cut to its upper 16 bits (an exact bf16); lo half = the rest
+                const uint32_t u0 = __float_as_uint(v0), u1 = __float_as_uint(v1);
+                const uint32_t u2 = __float_as_uint(v2), u3 = __float_as_uint(v3);
+                const uint32_t hiA = prmt(u0, u1, 0x7632u), hiB = prmt(u2, u3, 0x7632u);
+                const uint32_t loA = pack_bf16x2_rn(v0 - __uint_as_float(u0 & 0xffff0000u), v1 - __uint_as_float(u1 & 0xffff0000u));
+                const uint32_t loB = pack_bf16x2_rn(v2 - __uint_as_float(u2 & 0xffff0000u), v3 - __uint_as_float(u3 & 0xffff0000u));
+                pb[nt][0] = odd_col ? loA : hiA;
+                pb[nt][1] = odd_col ? loB : hiB;
             }
             // V pieces: slots [16g, 16g+16) of tokens t, t+4, t+8, t+12 of this row tile
             constexpr int VW = P / 2;      // words per token piece
             uint32_t vw[4][VW];
+            uint32_t ev[4];
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const uint8_t* pv = st + G_::VM_OFF + (mt * 16 + t + 4 * k) * ROW_M + g * (2 * P);
+                const uint8_t* pv = st + v_off + (mt * 16 + 4 * k) * ROW_M;
                 if (P == 4) {
                     uint2 x = *reinterpret_cast<const uint2*>(pv);
                     vw[k][0] = x.x; vw[k][1] = x.y;
@@ -481,27 +616,28 @@ __global__ void __launch_bounds__(kWarps * 32) decode_mma(DecodeArgs a) {
                     uint4 x = *reinterpret_cast<const uint4*>(pv);
                     vw[k][0] = x.x; vw[k][1] = x.y; vw[k][2] = x.z; vw[k][3] = x.w;
                 }
+                ev[k] = st[ve_off + (mt * 16 + 4 * k) * ROW_E];
             }
-            Wgt gA, gB;
-            {
-                const int eb = (16 * g) / N;
-                uint32_t s[4];
+            uint2 lv[4];
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const int row = mt * 16 + t + 4 * k;
-                    const uint32_t wv = weight_bf16<P>(st[G_::VE_OFF + row * ROW_E + eb]);
-                    s[k] = (row < n_live) ? wv : 0u;     // rows past the end contribute exactly zero
+            for (int k = 0; k < 4; ++k) lv[k] = lut[ev[k]];
+            if (!full) {       // rows past the end contribute exactly zero
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    if (mt * 16 + t + 4 * k >= n_live) lv[k] = make_uint2(0u, 0u);
+            }
+            const Wgt gA = make_wgt<P>(prmt(lv[0].x, lv[1].x, 0x7610u), prmt(lv[0].y, lv[1].y, 0x7610u));
+            const Wgt gB = make_wgt<P>(prmt(lv[2].x, lv[3].x, 0x7610u), prmt(lv[2].y, lv[3].y, 0x7610u));
+#pragma unroll
+            for (int r = 0; r < 8; r += 2) {
+                uint32_t xa[4], xb[4];
+                v_pairs2<P>(vw[0], vw[1], r, gA, sh, xa);
+                v_pairs2<P>(vw[2], vw[3], r, gB, sh, xb);
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    mma_bf16(o[nt][r], xa[0], xa[1], xb[0], xb[1], pb[nt][0], pb[nt][1]);
+                    mma_bf16(o[nt][r + 1], xa[2], xa[3], xb[2], xb[3], pb[nt][0], pb[nt][1]);
                 }
-                gA = make_wgt<P>(s[0] | (s[1] << 16));
-                gB = make_wgt<P>(s[2] | (s[3] << 16));
-            }
-#pragma unroll
-            for (int r = 0; r < 8; ++r) {
-                uint32_t a0, a1, a2, a3;
-                v_pairs<P>(vw[0], vw[1], r, gA, a0, a1);
-                v_pairs<P>(vw[2], vw[3], r, gB, a2, a3);
-#pragma unroll
-                for (int nt = 0; nt < NT; ++nt) mma_bf16(o[nt][r], a0, a1, a2, a3, pb[nt][0], pb[nt][1]);
             }
         }
 
@@ -550,7 +686,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s) {
     int dev = 0;
     KVBFP_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        KVBFP_CUDA(cudaFuncSetAttribute(decode_mma<P, N, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_::SMEM_BYTES));
+        KVBFP_CUDA(cudaFuncSetAttribute(decode_mma<P, N, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_::template smem_bytes<NT>()));
         attr_set[dev] = true;
     }
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
@@ -561,7 +697,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s) {
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma<P, N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(a);
+    decode_mma<P, N, NT><<<grid, kWarps * 32, G_::template smem_bytes<NT>(), s>>>(a);
     KVBFP_LAUNCH_CHECK("decode_mma");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;
