@@ -189,6 +189,33 @@ kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* q, kvbfp_dt
                                void* stream);
 
 /*
+ * kvbfp_decode_attn for callers that must not allocate device memory (the paper has no counterpart:
+ * this is a deployment aid, not a step of the method).  Who needs it: code that runs after a serving
+ * process has frozen its memory pool, plug-ins that are handed tensors but no allocator, and loops
+ * that cannot afford the device-wide synchronisation an allocation or a free may cause.  It computes
+ * exactly what kvbfp_decode_attn computes and takes the same arguments minus the workspace, which
+ * lives in a fixed array inside the library image instead.
+ *  - Limit: the array is kvbfp_static_scratch_bytes() = 32 MiB.  A geometry whose
+ *    kvbfp_decode_workspace_bytes() is larger is refused with KVBFP_ERR_WORKSPACE and nothing is
+ *    enqueued; use kvbfp_decode_attn with your own workspace then.  Every GPU on which the library is
+ *    loaded gives up those 32 MiB until the process exits.
+ *  - The call allocates nothing: no cudaMalloc, cudaFree or allocating library routine.
+ *  - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *    that device current) and keeps it; make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, which still holds the previous call's partial
+ *    results.  Nothing in it has to start at zero (each call writes every value it later reads), but
+ *    two calls that overlap on the GPU — different streams, or one stream while another still runs —
+ *    race on it and produce garbage.  Serialise them, or give the concurrent ones their own
+ *    workspace through kvbfp_decode_attn.
+ */
+size_t kvbfp_static_scratch_bytes(void);
+kvbfp_status kvbfp_decode_attn_static(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt,
+                                      int32_t n_q_heads, const int32_t* seq_lens,
+                                      int32_t max_len_hint, const int32_t* perm_k,
+                                      const int32_t* inv_perm_v, float softmax_scale,
+                                      int32_t q_mant_bits, float* out, uint32_t flags, void* stream);
+
+/*
  * One whole decode step for a caller whose new token lives in HOST memory (Sec. II-A: per step only
  * the new token's q, k, v are computed; the rest is read from the cache): copies k_new, v_new and q
  * to the device, appends the token (kvbfp_append with n_new = 1), runs kvbfp_decode_attn, copies the

@@ -23,7 +23,7 @@ EXPORTS = ["kvbfp_version", "kvbfp_status_string", "kvbfp_last_cuda_error", "kvb
            "kvbfp_calibrate", "kvbfp_fold_perm", "kvbfp_append", "kvbfp_dequant",
            "kvbfp_decode_workspace_bytes", "kvbfp_decode_attn", "kvbfp_device_status",
            "kvbfp_launch_count", "kvbfp_step_staging_bytes", "kvbfp_decode_step_host",
-           "kvbfp_profile_decode_events"]
+           "kvbfp_profile_decode_events", "kvbfp_static_scratch_bytes", "kvbfp_decode_attn_static"]
 
 
 class KvbfpError(RuntimeError):
@@ -92,6 +92,10 @@ def lib():
                                              C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_size_t,
                                              C.c_void_p, C.c_size_t, C.c_uint32, C.c_void_p]
         L.kvbfp_profile_decode_events.argtypes = [C.c_void_p, C.c_void_p]
+        L.kvbfp_static_scratch_bytes.restype = C.c_size_t
+        L.kvbfp_decode_attn_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int32,
+                                               C.c_void_p, C.c_void_p, C.c_float, C.c_int32, C.c_void_p,
+                                               C.c_uint32, C.c_void_p]
         _lib = L
     return _lib
 
@@ -266,3 +270,26 @@ def profile_decode_events(start=None, stop=None):
     a = None if start is None else C.c_void_p(start.cuda_event)
     b = None if stop is None else C.c_void_p(stop.cuda_event)
     _check(lib().kvbfp_profile_decode_events(a, b))
+
+
+def static_scratch_bytes():
+    return int(lib().kvbfp_static_scratch_bytes())
+
+
+def decode_attn_static(cache, q, seq_lens, perm_k=None, inv_perm_v=None, softmax_scale=0.0, max_len_hint=0,
+                       q_mant_bits=0, impl=DECODE_AUTO, chunk_tokens=0, out=None, stream=None):
+    """kvbfp_decode_attn_static: the same decode step for callers that cannot allocate device memory
+    (frozen memory pools, plug-ins without an allocator).  Its workspace is a fixed 32 MiB array inside
+    the library; larger geometries are refused.  Calls that overlap on the GPU race on that array.
+    ``out`` should be passed in by such callers; it is allocated here only as a convenience."""
+    q = _dev(q)
+    if out is None:
+        out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+    flags = impl | ((chunk_tokens // 128) << 8)
+    cs = cache.struct()
+    _check(lib().kvbfp_decode_attn_static(C.byref(cs), _ptr(q), _dt(q), q.shape[1],
+                                          _ptr(_dev(seq_lens, torch.int32)), max_len_hint,
+                                          _ptr(_dev(perm_k, torch.int32)), _ptr(_dev(inv_perm_v, torch.int32)),
+                                          float(softmax_scale), q_mant_bits, _ptr(_dev(out, torch.float32)), flags,
+                                          _stream(stream)))
+    return out
