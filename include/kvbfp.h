@@ -68,9 +68,11 @@ enum {
 
 /* Which decode kernel to run. */
 enum {
-    KVBFP_DECODE_AUTO = 0,  /* the tensor-core kernel                                          */
-    KVBFP_DECODE_SIMT = 1,  /* fp32 FMA on the plain ALUs, one query head at a time            */
-    KVBFP_DECODE_MMA = 2    /* grouped queries as the N operand of warp-level bf16 tensor MMAs */
+    KVBFP_DECODE_AUTO = 0,     /* the fastest tensor-core kernel for the format                       */
+    KVBFP_DECODE_SIMT = 1,     /* fp32 FMA on the plain ALUs, one query head at a time                */
+    KVBFP_DECODE_MMA = 2,      /* same as AUTO: grouped queries as the N operand of warp-level MMAs   */
+    KVBFP_DECODE_MMA_BF16 = 3  /* the generic bf16 tensor-core kernel (all mantissa widths); AUTO uses
+                                  it for 6 and 8 bits and the fp16 two-mantissas-per-element kernel for 4 */
 };
 /* Optional, or-ed into `flags`: tokens per sequence chunk (a multiple of 128; 0 = chosen by the
  * library from the batch size and the sequence bound). */

@@ -17,7 +17,7 @@ ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CAPACITY, ERR_WORKSPACE, ER
 F32, BF16 = 0, 1
 STAT_MAXABS, STAT_L2 = 0, 1
 FLAG_NONFINITE, FLAG_POSITION, FLAG_LEN_HINT, FLAG_WAIT_TIMEOUT = 1, 2, 4, 8
-DECODE_AUTO, DECODE_SIMT, DECODE_MMA = 0, 1, 2
+DECODE_AUTO, DECODE_SIMT, DECODE_MMA, DECODE_MMA_BF16 = 0, 1, 2, 3
 
 EXPORTS = ["kvbfp_version", "kvbfp_status_string", "kvbfp_last_cuda_error", "kvbfp_plane_bytes",
            "kvbfp_calibrate", "kvbfp_fold_perm", "kvbfp_append", "kvbfp_dequant",

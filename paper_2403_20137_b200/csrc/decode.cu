@@ -7,11 +7,15 @@
 namespace kvbfp {
 namespace {
 
-// One warp per (batch, query head): out = sum_i 2^(m_i - m) o_i / sum_i 2^(m_i - m) l_i.
+// One warp per (batch, query head): out = sum_i 2^(m_i - m) o_i / sum_i 2^(m_i - m) l_i over the partial
+// results of the row.  n_warps == 0: every chunk that holds tokens has its own partial.  n_warps > 0:
+// the items (pair-major chunks) were cut into n_warps contiguous ranges and each range wrote one partial
+// per (batch, kv head) it touches, at the slot of the first chunk it covers there; the same integer
+// arithmetic as in the kernel finds those slots.
 __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ partials, const int32_t* __restrict__ seq_lens,
                                                  const int32_t* __restrict__ inv_perm_v, float* __restrict__ out,
                                                  int n_rows, int n_q_heads, int group, int n_chunks, int chunk,
-                                                 int len_cap) {
+                                                 int len_cap, int n_warps, long long n_items) {
     constexpr int D = kHeadDim;
     __shared__ float so[4][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -22,20 +26,28 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
     len = len < 0 ? 0 : (len > len_cap ? len_cap : len);
     const int nc = (len + chunk - 1) / chunk;        // chunks that hold tokens
     const float* base = partials + (int64_t)row * n_chunks * kPartStride;
-    float m = -INFINITY;
-    for (int i = lane; i < nc; i += 32) m = fmaxf(m, base[(int64_t)i * kPartStride + D]);
-#pragma unroll
-    for (int off = 16; off; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    const long long first = ((long long)b * (n_q_heads / group) + hq / group) * n_chunks;   // first item of the pair
+    float m = -INFINITY, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    float l = 0.f;
-    for (int i = 0; i < nc; ++i) {
+    for (int i = 0; i < nc;) {
         const float* p = base + (int64_t)i * kPartStride;
-        const float w = exp2f(p[D] - m);
+        const float mi = p[D], li = p[D + 1];
         const float4 o = *reinterpret_cast<const float4*>(p + lane * 4);
-        acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
-        l += w * p[D + 1];
+        const float mn = fmaxf(m, mi);
+        const float a1 = (m == -INFINITY) ? 0.f : exp2f(m - mn), a2 = (mi == -INFINITY) ? 0.f : exp2f(mi - mn);
+        acc.x = acc.x * a1 + a2 * o.x; acc.y = acc.y * a1 + a2 * o.y;
+        acc.z = acc.z * a1 + a2 * o.z; acc.w = acc.w * a1 + a2 * o.w;
+        l = l * a1 + a2 * li;
+        m = mn;
+        if (n_warps == 0) {
+            ++i;
+        } else {                                     // next partial of the pair: where the next range starts
+            const long long item = first + i;
+            const long long w = ((item + 1) * n_warps - 1) / n_items;      // range that holds this item
+            i = (int)(((w + 1) * n_items) / n_warps - first);
+        }
     }
-    const float inv = (nc > 0 && l > 0.f) ? 1.f / l : 0.f;
+    const float inv = (l > 0.f) ? 1.f / l : 0.f;
     float* dst = out + (int64_t)row * D;
     if (!inv_perm_v) {
         *reinterpret_cast<float4*>(dst + lane * 4) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
@@ -63,7 +75,9 @@ void profile_events(cudaEvent_t* start, cudaEvent_t* stop) {
 size_t qfrag_bytes(const kvbfp_format& f, int n_q_heads) {
     const int group = n_q_heads / f.n_kv_heads;
     const int nt = (group + 3) / 4;                  // four query heads per 8-column MMA tile
-    return (size_t)f.batch * f.n_kv_heads * nt * 8 * 32 * 2 * sizeof(uint32_t);
+    const size_t frag = (size_t)f.batch * f.n_kv_heads * nt * 8 * 32 * 2 * sizeof(uint32_t);
+    const size_t qexp = ((size_t)f.batch * n_q_heads * sizeof(int32_t) + 255) & ~(size_t)255;   // per-query exponents
+    return frag + qexp;
 }
 
 }  // namespace kvbfp
@@ -94,7 +108,7 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
     if (q_mant_bits != 0 && q_mant_bits != 8) return KVBFP_ERR_UNSUPPORTED;
     if (max_len_hint < 0 || !(softmax_scale >= 0.f) || isinf(softmax_scale)) return KVBFP_ERR_INVALID_ARG;
     const uint32_t impl = flags & 0xffu, chunk_units = (flags >> 8) & 0xfffu;
-    if (impl > KVBFP_DECODE_MMA || (flags >> 20)) return KVBFP_ERR_INVALID_ARG;
+    if (impl > KVBFP_DECODE_MMA_BF16 || (flags >> 20)) return KVBFP_ERR_INVALID_ARG;
     const void* ptrs[] = {cache->k_mant, cache->k_exp, cache->v_mant, cache->v_exp, q, out, workspace, perm_k, inv_perm_v};
     for (const void* p : ptrs)
         if (p && !aligned16(p)) return KVBFP_ERR_ALIGNMENT;
@@ -116,9 +130,12 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
 
     // Sequence chunking: enough independent (batch, kv head, chunk) items to keep every warp slot of
     // the machine busy for a few rounds, chunks in multiples of kMinChunk tokens.
+    const bool use_mma4 = impl != KVBFP_DECODE_SIMT && impl != KVBFP_DECODE_MMA_BF16 && f.mant_bits == 4;
     int chunk;
     if (chunk_units) {
         chunk = (int)chunk_units * kMinChunk;
+    } else if (use_mma4) {
+        chunk = kMinChunk;      // the persistent kernel balances by item count: finest items, one partial per range
     } else {
         const int64_t pairs = (int64_t)f.batch * f.n_kv_heads;
         const int64_t target_items = 148 * 16 * 4;
@@ -135,11 +152,15 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
     a.mulhi4 = 1u << 28; a.mulhi8 = 1u << 24; a.mulhi12 = 1u << 20;
 
     cudaStream_t s = (cudaStream_t)stream;
-    st = (impl == KVBFP_DECODE_SIMT) ? launch_decode_simt(a, s) : launch_decode_mma(a, s);
+    int n_warps = 0;
+    if (impl == KVBFP_DECODE_SIMT) st = launch_decode_simt(a, s);
+    else if (use_mma4) st = launch_decode_mma4(a, s, &n_warps);
+    else st = launch_decode_mma(a, s);
     if (st != KVBFP_OK) return st;
     const int n_rows = f.batch * n_q_heads;
     lse_merge<<<(n_rows + 3) / 4, 128, 0, s>>>(a.partials, seq_lens, inv_perm_v, out, n_rows, n_q_heads, group,
-                                              a.n_chunks, a.chunk, a.len_cap);
+                                              a.n_chunks, a.chunk, a.len_cap, n_warps,
+                                              (long long)f.batch * f.n_kv_heads * a.n_chunks);
     KVBFP_LAUNCH_CHECK("lse_merge");
     return KVBFP_OK;
 }

@@ -33,7 +33,9 @@ struct DecodeArgs {
 };
 
 kvbfp_status launch_decode_simt(const DecodeArgs& a, cudaStream_t s);
-kvbfp_status launch_decode_mma(const DecodeArgs& a, cudaStream_t s);
+kvbfp_status launch_decode_mma(const DecodeArgs& a, cudaStream_t s);    // bf16, every mantissa width
+// fp16, 4-bit mantissas, persistent: *n_warps receives the number of warps the items were split over
+kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, int* n_warps);
 size_t qfrag_bytes(const kvbfp_format& f, int n_q_heads);
 // Events the caller asked to have recorded around the main decode kernel (nullptr = none).
 void profile_events(cudaEvent_t* start, cudaEvent_t* stop);

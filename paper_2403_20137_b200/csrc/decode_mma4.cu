@@ -1,0 +1,620 @@
+// Decode attention over a 4-bit BFP cache with fp16 tensor-core MMAs, two mantissas per operand element
+// (Sec. III par. 2 of the paper: keys are read back from the cache and multiplied with pi(q);
+// Sec. II-B: a block's values are integer mantissas times one power of two).
+//
+// Work split.  The (batch, kv head, 128-token chunk) items are laid out pair-major and cut into one
+// contiguous range per resident warp; the kernel is persistent (one launch fills the machine once).
+// A warp walks its range as "runs" -- the chunks of one (batch, kv head) that fall into the range --
+// keeping one set of accumulators per run and writing one partial result per run, at the slot of the
+// run's first chunk.  Each warp has a private ring of shared-memory stages filled by 1-D bulk
+// asynchronous copies (lanes 0..3 issue one span each, an mbarrier per stage counts the bytes); the
+// copies run ahead across run boundaries, so a new run starts with its first tiles already on chip.
+// There is no block-wide barrier in the loop and no cluster multicast.
+//
+// Unpacking is what limits this kernel (integer-pipe instructions, not memory).  A packed byte holds
+// two mantissas; with the sign bits flipped it is B = 16*(M_hi+8) + (M_lo+8).  fp16 has a 10-bit
+// fraction, so the whole byte can be put under the bits of 1024.0 with one byte permute: the element
+// 1024 + B.  A second element with the high nibble masked away and bit 7 set, 1024 + 128 + (M_lo+8),
+// comes from one logic op.  One f16x2 fma per register with the block's power of two removes the
+// common bias 1160 and applies the weight, exactly:
+//     kind 1:  (16*M_hi + M_lo) * w        kind 2:  M_lo * w
+// The two mantissas are then separated by linearity instead of by shifts:
+//   scores:  q_hi*M_hi + q_lo*M_lo = (q_hi/16) * kind1 + (q_lo - q_hi/16) * kind2, so the query
+//            fragment simply carries those two coefficients at the two k positions;
+//   output:  the row of kind 1 accumulates 16*o_hi + o_lo and the row of kind 2 accumulates o_lo;
+//            o_hi = (row1 - row2)/16 once, when the run's partial result is written.
+//
+// Range.  fp16 cannot hold 2^e for every exponent byte, so each run first takes the largest K and V
+// exponent byte of its rows (D_k, D_v) and uses the weights 2^(e - D + 5): the largest block gets
+// 2^5 (the bias product 1160 * 2^5 still fits fp16), blocks more than 2^29 below the largest one of
+// the run are flushed to zero (their contribution is below 2^-29 of it), and the common factor
+// 2^(D - 134) is applied in fp32 to the scores and to the partial output.  The weights come from a
+// shared-memory table addressed by exponent byte from a per-run base, so the subtraction costs
+// nothing.  q and the softmax weights are carried as (hi, lo) fp16 pairs (q after a per-head
+// power-of-two normalisation), accumulation is fp32.
+#include <math.h>
+
+#include <type_traits>
+
+#include "decode.cuh"
+#include "ptx.cuh"
+
+namespace kvbfp {
+namespace {
+
+#ifndef KVBFP4_WARPS
+#define KVBFP4_WARPS 4
+#endif
+#ifndef KVBFP4_MT
+#define KVBFP4_MT 4
+#endif
+#ifndef KVBFP4_STAGES
+#define KVBFP4_STAGES 2
+#endif
+#ifndef KVBFP4_MIN_CTAS
+#define KVBFP4_MIN_CTAS 1
+#endif
+
+constexpr int kWarps = KVBFP4_WARPS;
+constexpr int kMT = KVBFP4_MT;          // 16-token MMA row tiles per stage
+constexpr int kTile = 16 * kMT;         // tokens per stage
+constexpr int kStages = KVBFP4_STAGES;
+constexpr int D = kHeadDim;
+constexpr int ROW_M = D / 2;            // 64 bytes of mantissas per token row
+constexpr int kTopShift = 5;            // weight of the run's largest block is 2^kTopShift
+constexpr int kLutEntries = 512;        // index = exponent byte - D + 255, D = largest valid exponent byte
+
+constexpr uint32_t kMagic = 0x64646464u;        // 0x64 = high byte of fp16 1024.0
+constexpr uint32_t kBias = 0xE488E488u;         // fp16 -1160.0 twice
+constexpr uint32_t kFlip = 0x88888888u;         // flips the sign bit of every 4-bit field: M -> M + 8
+
+// fp16 bit pattern of 2^j for j in [-24, 15], 0 below.
+__device__ __forceinline__ uint32_t pow2_f16(int j) {
+    if (j >= -14) return (uint32_t)(j + 15) << 10;
+    if (j >= -24) return 1u << (j + 24);
+    return 0u;
+}
+
+// 2^ex as a float for any ex that the product with an ordinary number keeps in range (two exact factors).
+__device__ __forceinline__ float pow2_split(float x, int ex) {
+    const int e1 = ex / 2, e2 = ex - e1;
+    return (x * exp2f((float)e1)) * exp2f((float)e2);
+}
+
+// Byte `byte` (0..63) of a row: low nibble = slot 2*byte, high nibble = slot 2*byte+1.
+// K side, k position kk (0..3 = k 2t, 2t+1, 2t+8, 2t+9) of k-step ks for lane column t:
+//   byte = 16t + 4(ks/2) + 2(ks%2) + (kk%2), kind 1 (whole byte) for kk < 2, kind 2 (low nibble) for kk >= 2.
+
+// ------------------------------------------------------------------ query fragments
+// One warp per (batch, kv head, n-tile).  Writes, in MMA B-fragment order, the (hi, lo) fp16 halves of
+// the coefficients c1 = q_hi/16 (whole byte) and c2 = q_lo - q_hi/16 (low nibble), normalised per query
+// head by a power of two 2^qe, and qe itself.
+__global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t* qexp) {
+    const int N = a.fmt.block;
+    const int lane = threadIdx.x, gp = lane >> 2, tp = lane & 3;
+    const int item = blockIdx.x;
+    const int nt = item % NT, hk = (item / NT) % a.fmt.n_kv_heads, b = item / NT / a.fmt.n_kv_heads;
+    const int G = a.n_q_heads / a.fmt.n_kv_heads;
+    __shared__ float sq[4][D];       // pi(q) of the four query heads of this n-tile, then the coefficients
+    __shared__ int sqe[4];
+    for (int i = lane; i < 4 * D; i += 32) {
+        const int qq = 4 * nt + i / D, slot = i % D;
+        float v = 0.f;
+        if (qq < G) {
+            const int ch = a.perm_k ? (a.perm_k[hk * D + slot] & (D - 1)) : slot;
+            const int64_t idx = ((int64_t)b * a.n_q_heads + hk * G + qq) * D + ch;
+            v = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
+        }
+        sq[i / D][slot] = v;
+    }
+    __syncwarp();
+    if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
+        const int nblk = D / N;
+        for (int i = lane; i < 4 * nblk; i += 32) {
+            float* blk = &sq[i / nblk][(i % nblk) * N];
+            uint32_t am = 0;
+            for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(blk[j]) & 0x7fffffffu);
+            int e8 = (int)(am >> 23);
+            if (e8 == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e8 = 254; }
+            const int k = 127 - e8 + 6, k1 = k >> 1, k2 = k - k1;
+            const float w = unit_weight(e8, 8);
+            for (int j = 0; j < N; ++j) {
+                float tv = (blk[j] * pow2i(k1)) * pow2i(k2);
+                blk[j] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * w;
+            }
+        }
+        __syncwarp();
+    }
+    // coefficients in place: slot 2j <- c2 (low nibble), slot 2j+1 <- c1 (whole byte); per-head exponent.
+    // Lane l owns bytes l and l + 32 (slots 2l, 2l+1, 2l+64, 2l+65).
+    for (int qq = 0; qq < 4; ++qq) {
+        const float c1a = sq[qq][2 * lane + 1] * 0.0625f, c2a = sq[qq][2 * lane] - c1a;
+        const float c1b = sq[qq][2 * lane + 65] * 0.0625f, c2b = sq[qq][2 * lane + 64] - c1b;
+        uint32_t am = max(max(__float_as_uint(c1a) & 0x7fffffffu, __float_as_uint(c2a) & 0x7fffffffu),
+                          max(__float_as_uint(c1b) & 0x7fffffffu, __float_as_uint(c2b) & 0x7fffffffu));
+#pragma unroll
+        for (int off = 16; off; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+        int e = (int)(am >> 23);
+        if (e == 255) { if (lane == 0) raise_flag(a.status, KVBFP_FLAG_NONFINITE); e = 254; }
+        const int qe = (am == 0) ? 0 : e - 126;               // |c| * 2^-qe < 1
+        // scale by 2^-qe in two exact steps (qe in [-126, 128])
+        const int h1 = (-qe) / 2, h2 = (-qe) - h1;
+        const float f1 = pow2i(h1), f2 = pow2i(h2);
+        sq[qq][2 * lane] = (c2a * f1) * f2;       sq[qq][2 * lane + 1] = (c1a * f1) * f2;
+        sq[qq][2 * lane + 64] = (c2b * f1) * f2;  sq[qq][2 * lane + 65] = (c1b * f1) * f2;
+        if (lane == 0) sqe[qq] = qe;
+    }
+    __syncwarp();
+    if (lane < 4 && 4 * nt + lane < G) qexp[(int64_t)b * a.n_q_heads + hk * G + 4 * nt + lane] = sqe[lane];
+
+    const int qi = 4 * nt + (gp >> 1), part = gp & 1;
+    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32 * 2);
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) {
+        uint32_t reg[2];
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) {         // rr = 0: kind 1 (k 2t, 2t+1); rr = 1: kind 2 (k 2t+8, 2t+9)
+            uint32_t h[2];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int byte = 16 * tp + 4 * (ks >> 1) + 2 * (ks & 1) + e;
+                const float v = sq[gp >> 1][2 * byte + (rr == 0 ? 1 : 0)];
+                const __half hi = __float2half_rn(v);
+                __half out = part ? __float2half_rn(v - __half2float(hi)) : hi;
+                if (qi >= G) out = __ushort_as_half(0);
+                h[e] = __half_as_ushort(out);
+            }
+            reg[rr] = h[0] | (h[1] << 16);
+        }
+        const int wd = 2 * ks;
+        dst[((wd >> 2) * 32 + lane) * 4 + (wd & 3)] = reg[0];
+        dst[((wd >> 2) * 32 + lane) * 4 + (wd & 3) + 1] = reg[1];
+    }
+}
+
+// ------------------------------------------------------------------ main kernel
+template <int N>
+struct Geo4 {
+    static constexpr int ROW_E = D / N;
+    static constexpr int KM_OFF = 0;
+    static constexpr int VM_OFF = kTile * ROW_M;
+    static constexpr int KE_OFF = 2 * kTile * ROW_M;
+    static constexpr int VE_OFF = KE_OFF + kTile * ROW_E;
+    static constexpr int STAGE_BYTES = 2 * kTile * (ROW_M + ROW_E);
+    static constexpr int WARP_BYTES = kStages * STAGE_BYTES;
+    static constexpr int LUT_OFF = kWarps * WARP_BYTES;                 // uint2[kLutEntries]
+    static constexpr int BAR_OFF = LUT_OFF + kLutEntries * 8;
+    static constexpr int SMEM_BYTES = BAR_OFF + kWarps * kStages * 8;
+};
+
+// Largest of the first `bytes` bytes of a 16-byte-aligned span in global memory, over the warp.  Whole
+// 16-byte vectors are loaded (the span is padded to a multiple of 16 inside the plane); bytes past
+// `bytes` are masked out.
+__device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int lane) {
+    uint32_t m = 0;
+    const uint4* v = reinterpret_cast<const uint4*>(p);
+    for (int i = lane; i < ((bytes + 15) >> 4); i += 32) {
+        uint4 x = __ldg(v + i);
+        const int left = bytes - 16 * i;             // valid bytes in this vector (may exceed 16)
+        if (left < 16) {
+            uint32_t w[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int r = left - 4 * k;
+                w[k] = r >= 4 ? w[k] : (r <= 0 ? 0u : (w[k] & ((1u << (8 * r)) - 1u)));
+            }
+            x = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        m = vmaxu4(vmaxu4(m, x.x), vmaxu4(x.y, vmaxu4(x.z, x.w)));
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1) m = vmaxu4(m, __shfl_xor_sync(0xffffffffu, m, off));
+    m = vmaxu4(m, m >> 16);
+    m = vmaxu4(m, m >> 8);
+    return (int)(m & 0xffu);
+}
+
+// The chunks of one (batch, kv head) that fall into a warp's item range.
+struct Run {
+    int b, hk;
+    int chunk0;        // first chunk: its slot receives the partial result
+    int n_items;       // chunks covered (>= 1)
+    int n_tok;         // tokens that exist in them (0: nothing to do)
+    int n_tiles;
+    int64_t row0;      // first row in the planes
+};
+
+template <int N, int NT>
+__global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(DecodeArgs a, const int32_t* __restrict__ qexp) {
+    using G_ = Geo4<N>;
+    constexpr int ROW_E = G_::ROW_E;
+    constexpr int NBK = (N == 16) ? 2 : 1;            // blocks inside a K lane chunk of 32 slots
+    extern __shared__ __align__(128) uint8_t smem[];
+
+    // weight table: entry i = (2^(i - 255 + kTopShift) twice as f16x2, the same times -1160); entries
+    // above 255 belong to rows that are masked later (past the end of the run) and only have to exist
+    uint2* lut = reinterpret_cast<uint2*>(smem + G_::LUT_OFF);
+    for (int i = threadIdx.x; i < kLutEntries; i += kWarps * 32) {
+        const uint32_t s2 = (i <= 255 ? pow2_f16(i - 255 + kTopShift) : 0u) * 0x00010001u;
+        lut[i] = make_uint2(s2, mul_f16x2(s2, kBias));
+    }
+    __syncthreads();
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
+    const int64_t n_items = (int64_t)a.fmt.batch * Hkv * a.n_chunks;
+    const int64_t wglob = (int64_t)blockIdx.x * kWarps + warp, wtot = (int64_t)gridDim.x * kWarps;
+    const int64_t i0 = wglob * n_items / wtot, i1 = (wglob + 1) * n_items / wtot;     // this warp's items
+    if (i0 >= i1) return;
+
+    auto get_run = [&](int64_t it) -> Run {
+        Run r;
+        const int64_t pair = it / a.n_chunks;
+        r.chunk0 = (int)(it - pair * a.n_chunks);
+        r.hk = (int)(pair % Hkv);
+        r.b = (int)(pair / Hkv);
+        const int64_t left = i1 - it;
+        r.n_items = (int)(left < (int64_t)(a.n_chunks - r.chunk0) ? left : (int64_t)(a.n_chunks - r.chunk0));
+        int len = a.seq_lens[r.b];
+        if (len > a.fmt.max_seq || len < 0) {
+            if (lane == 0 && r.chunk0 == 0 && r.hk == 0) raise_flag(a.status, KVBFP_FLAG_POSITION);
+            len = len < 0 ? 0 : a.fmt.max_seq;
+        }
+        if (len > a.len_cap) {
+            if (lane == 0 && r.chunk0 == 0 && r.hk == 0) raise_flag(a.status, KVBFP_FLAG_LEN_HINT);
+            len = a.len_cap;
+        }
+        const int tok0 = r.chunk0 * a.chunk;
+        const int64_t tok1 = (int64_t)(r.chunk0 + r.n_items) * a.chunk;
+        r.n_tok = max(0, (int)min((int64_t)len, tok1) - tok0);
+        r.n_tiles = (r.n_tok + kTile - 1) / kTile;
+        r.row0 = pair * a.fmt.max_seq + tok0;
+        return r;
+    };
+
+    uint8_t* wsm = smem + warp * G_::WARP_BYTES;
+    const uint32_t wsm_u32 = smem_u32(wsm);
+    const uint32_t bar0 = smem_u32(smem + G_::BAR_OFF + warp * kStages * 8);
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) mbar_init(bar0 + 8 * s, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+
+    // ---- producer: lanes 0..3 each own one of the four spans of a stage (K mantissas, V mantissas,
+    // K exponents, V exponents).  The cursor (p_run, p_tile) runs ahead of the consumer by kStages tiles.
+    const uint8_t* my_base = lane == 0 ? a.k_mant : lane == 1 ? a.v_mant : lane == 2 ? a.k_exp : a.v_exp;
+    const int my_row_bytes = (lane < 2) ? ROW_M : ROW_E;
+    const uint32_t my_dst = wsm_u32 + (lane == 0 ? G_::KM_OFF : lane == 1 ? G_::VM_OFF : lane == 2 ? G_::KE_OFF : G_::VE_OFF);
+    int64_t p_next = i0;
+    Run pr;
+    pr.n_tiles = 0;
+    int p_tile = 0;
+    auto issue_next = [&](int stage) {
+        while (p_tile >= pr.n_tiles) {               // next run that has tokens
+            if (p_next >= i1) return;
+            pr = get_run(p_next);
+            p_next += pr.n_items;
+            p_tile = 0;
+        }
+        if (lane < 4) {
+            const int off = p_tile * kTile;
+            const int rows = min(kTile, ((pr.n_tok + 15) & ~15) - off);    // whole 16-token groups; stays below max_seq
+            const uint32_t bar = bar0 + 8 * stage;
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(2 * rows * (ROW_M + ROW_E)));
+            __syncwarp(0xfu);
+            bulk_g2s(my_dst + stage * G_::STAGE_BYTES, my_base + (pr.row0 + off) * my_row_bytes, rows * my_row_bytes, bar);
+        }
+        ++p_tile;
+    };
+    for (int s = 0; s < kStages; ++s) issue_next(s);
+
+    // per-lane byte offsets inside a stage
+    const int k_off = G_::KM_OFF + g * ROW_M + t * 16;
+    const int ke_off = G_::KE_OFF + g * ROW_E + ((N == 16) ? 2 * t : (N == 32) ? t : (N == 64) ? (t >> 1) : 0);
+    const int v_off = G_::VM_OFF + t * ROW_M + g * 8;
+    const int ve_off = G_::VE_OFF + t * ROW_E + (16 * g) / N;
+    const int src_lo = 4 * t + (g >> 1), src_hi = 4 * (t + 4) + (g >> 1);
+    const bool odd_col = (g & 1) != 0;
+
+    int stage = 0;
+    uint32_t parity = 0;
+    bool timed_out = false;
+
+    for (int64_t c_next = i0; c_next < i1 && !timed_out;) {
+        const Run cr = get_run(c_next);
+        c_next += cr.n_items;
+        if (cr.n_tok == 0) continue;
+
+        // ---- run set-up: exponent references, query fragments, score factors ------------------
+        const int dk = warp_max_byte(a.k_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
+        const int dv = warp_max_byte(a.v_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
+        const uint2* lutk = lut + (255 - dk);
+        const uint2* lutv = lut + (255 - dv);
+        uint2 qf[NT][8];
+        float kfac[NT];
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(a.qfrag) + (((int64_t)cr.b * Hkv + cr.hk) * NT) * (4 * 32);
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint4 v = __ldg(src + (nt * 4 + j) * 32 + lane);
+                    qf[nt][2 * j] = make_uint2(v.x, v.y);
+                    qf[nt][2 * j + 1] = make_uint2(v.z, v.w);
+                }
+                const int qi = 4 * nt + t;
+                const int qe = (qi < Gq) ? qexp[(int64_t)cr.b * a.n_q_heads + cr.hk * Gq + qi] : 0;
+                kfac[nt] = pow2_split(a.scale_log2e, dk - 129 - kTopShift + qe);
+            }
+        }
+        float o[NT][8][4];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int r = 0; r < 8; ++r)
+#pragma unroll
+                for (int k = 0; k < 4; ++k) o[nt][r][k] = 0.f;
+        float m_run[NT], l_run[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) { m_run[nt] = -INFINITY; l_run[nt] = 0.f; }
+
+        // one stage of kTile tokens; FULL = every row of the tile exists
+        auto tile_body = [&](const uint8_t* st, int n_live, auto full_tag) {
+            constexpr bool FULL = decltype(full_tag)::value;
+            // ---- scores ---------------------------------------------------------
+            float sc[kMT][NT][2];
+#pragma unroll
+            for (int mt = 0; mt < kMT; ++mt) {
+                if (!FULL && mt * 16 >= n_live) {
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = -INFINITY;
+                    continue;
+                }
+                const uint4 xa = *reinterpret_cast<const uint4*>(st + k_off + mt * 16 * ROW_M);
+                const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off + (mt * 16 + 8) * ROW_M);
+                const uint32_t wa[4] = {xa.x ^ kFlip, xa.y ^ kFlip, xa.z ^ kFlip, xa.w ^ kFlip};      // sign bits -> offsets
+                const uint32_t wb[4] = {xb.x ^ kFlip, xb.y ^ kFlip, xb.z ^ kFlip, xb.w ^ kFlip};
+                uint2 la[NBK], lb[NBK];
+#pragma unroll
+                for (int k = 0; k < NBK; ++k) {
+                    la[k] = lutk[st[ke_off + mt * 16 * ROW_E + k]];
+                    lb[k] = lutk[st[ke_off + (mt * 16 + 8) * ROW_E + k]];
+                }
+                float acc[NT][2][4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int kb = (NBK == 2) ? (i >> 1) : 0;
+                    // bytes 4i..4i+3 of the lane chunk: kind 1 by byte permute, kind 2 by one logic op
+                    const uint32_t a1_01 = prmt(wa[i], kMagic, 0x4140u), a1_23 = prmt(wa[i], kMagic, 0x4342u);
+                    const uint32_t b1_01 = prmt(wb[i], kMagic, 0x4140u), b1_23 = prmt(wb[i], kMagic, 0x4342u);
+                    const uint32_t a2_01 = lop3<0x6A>(a1_01, 0xFF0FFF0Fu, 0x00800080u), a2_23 = lop3<0x6A>(a1_23, 0xFF0FFF0Fu, 0x00800080u);
+                    const uint32_t b2_01 = lop3<0x6A>(b1_01, 0xFF0FFF0Fu, 0x00800080u), b2_23 = lop3<0x6A>(b1_23, 0xFF0FFF0Fu, 0x00800080u);
+                    const uint32_t A0 = fma_f16x2(a1_01, la[kb].x, la[kb].y), A1 = fma_f16x2(b1_01, lb[kb].x, lb[kb].y);
+                    const uint32_t A2 = fma_f16x2(a2_01, la[kb].x, la[kb].y), A3 = fma_f16x2(b2_01, lb[kb].x, lb[kb].y);
+                    const uint32_t B0 = fma_f16x2(a1_23, la[kb].x, la[kb].y), B1 = fma_f16x2(b1_23, lb[kb].x, lb[kb].y);
+                    const uint32_t B2 = fma_f16x2(a2_23, la[kb].x, la[kb].y), B3 = fma_f16x2(b2_23, lb[kb].x, lb[kb].y);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint2 q0 = qf[nt][2 * i], q1 = qf[nt][2 * i + 1];
+                        if (i == 0) {
+                            mma_f16_first(acc[nt][0], A0, A1, A2, A3, q0.x, q0.y);
+                            mma_f16_first(acc[nt][1], B0, B1, B2, B3, q1.x, q1.y);
+                        } else {
+                            mma_f16(acc[nt][0], A0, A1, A2, A3, q0.x, q0.y);
+                            mma_f16(acc[nt][1], B0, B1, B2, B3, q1.x, q1.y);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    sc[mt][nt][0] = ((acc[nt][0][0] + acc[nt][0][1]) + (acc[nt][1][0] + acc[nt][1][1])) * kfac[nt];
+                    sc[mt][nt][1] = ((acc[nt][0][2] + acc[nt][0][3]) + (acc[nt][1][2] + acc[nt][1][3])) * kfac[nt];
+                }
+                if (!FULL) {       // select, not arithmetic: rows past the end may hold anything
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        if (mt * 16 + g >= n_live) sc[mt][nt][0] = -INFINITY;
+                        if (mt * 16 + g + 8 >= n_live) sc[mt][nt][1] = -INFINITY;
+                    }
+                }
+            }
+
+            // ---- running softmax (reference point moves only in big steps) ------
+            bool grow = false;
+            float tmax[NT];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) {
+                float mx = -INFINITY;
+#pragma unroll
+                for (int mt = 0; mt < kMT; ++mt) mx = fmaxf(mx, fmaxf(sc[mt][nt][0], sc[mt][nt][1]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                tmax[nt] = mx;
+                grow |= mx > m_run[nt] + 8.f;
+            }
+            if (__any_sync(0xffffffffu, grow)) {
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const float m_new = fmaxf(m_run[nt], tmax[nt]);
+                    const float alpha = (m_run[nt] == -INFINITY) ? 0.f : ex2_approx(m_run[nt] - m_new);
+                    m_run[nt] = m_new;
+                    l_run[nt] *= alpha;
+#pragma unroll
+                    for (int r = 0; r < 8; ++r)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) o[nt][r][k] *= alpha;
+                }
+            }
+
+            // ---- P.V ------------------------------------------------------------
+#pragma unroll
+            for (int mt = 0; mt < kMT; ++mt) {
+                if (!FULL && mt * 16 >= n_live) continue;
+                // softmax weights of this lane's tokens (g and g+8), then the B fragment of P^T for lane (g, t):
+                // column g = (query g/2, half g%2); tokens t, t+4 | t+8, t+12
+                uint32_t pb[NT][2];
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const float p0 = ex2_approx(sc[mt][nt][0] - m_run[nt]);
+                    const float p1 = ex2_approx(sc[mt][nt][1] - m_run[nt]);
+                    l_run[nt] += p0 + p1;
+                    const float v0 = __shfl_sync(0xffffffffu, p0, src_lo);   // token t
+                    const float v1 = __shfl_sync(0xffffffffu, p0, src_hi);   // token t+4
+                    const float v2 = __shfl_sync(0xffffffffu, p1, src_lo);   // token t+8
+                    const float v3 = __shfl_sync(0xffffffffu, p1, src_hi);   // token t+12
+                    // hi half = the value cut to 11 significant bits (exact in fp16); lo half = the rest
+                    const float h0 = __uint_as_float(__float_as_uint(v0) & 0xffffe000u);
+                    const float h1 = __uint_as_float(__float_as_uint(v1) & 0xffffe000u);
+                    const float h2 = __uint_as_float(__float_as_uint(v2) & 0xffffe000u);
+                    const float h3 = __uint_as_float(__float_as_uint(v3) & 0xffffe000u);
+                    pb[nt][0] = odd_col ? pack_f16x2_rn(v0 - h0, v1 - h1) : pack_f16x2_rn(h0, h1);
+                    pb[nt][1] = odd_col ? pack_f16x2_rn(v2 - h2, v3 - h3) : pack_f16x2_rn(h2, h3);
+                }
+                // V pieces: bytes [8g, 8g+8) (slots 16g..16g+15) of tokens t, t+4, t+8, t+12 of this row tile
+                uint2 vw[4];
+                uint2 lv[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    vw[k] = *reinterpret_cast<const uint2*>(st + v_off + (mt * 16 + 4 * k) * ROW_M);
+                    lv[k] = lutv[st[ve_off + (mt * 16 + 4 * k) * ROW_E]];
+                }
+                if (!FULL) {       // rows past the end contribute exactly zero
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        if (mt * 16 + t + 4 * k >= n_live) lv[k] = make_uint2(0u, 0u);
+                }
+                const uint32_t sA = prmt(lv[0].x, lv[1].x, 0x7610u), cA = prmt(lv[0].y, lv[1].y, 0x7610u);
+                const uint32_t sB = prmt(lv[2].x, lv[3].x, 0x7610u), cB = prmt(lv[2].y, lv[3].y, 0x7610u);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {         // byte pair (2x, 2x+1) of the lane's eight bytes
+                    const uint32_t wA0 = (x < 2) ? vw[0].x : vw[0].y, wA1 = (x < 2) ? vw[1].x : vw[1].y;
+                    const uint32_t wB0 = (x < 2) ? vw[2].x : vw[2].y, wB1 = (x < 2) ? vw[3].x : vw[3].y;
+                    const uint32_t sel = (x & 1) ? 0x7632u : 0x5410u;
+                    // [tok.b, tok.b', tok'.b, tok'.b'] with the sign bits turned into offsets
+                    const uint32_t XA = prmt(wA0, wA1, sel) ^ kFlip, XB = prmt(wB0, wB1, sel) ^ kFlip;
+                    // kind 1 for the even byte by mask-or, for the odd byte by byte permute; kind 2 from kind 1
+                    const uint32_t a1e = lop3<0xEA>(XA, 0x00FF00FFu, 0x64006400u), a1o = prmt(XA, kMagic, 0x4341u);
+                    const uint32_t b1e = lop3<0xEA>(XB, 0x00FF00FFu, 0x64006400u), b1o = prmt(XB, kMagic, 0x4341u);
+                    const uint32_t a2e = lop3<0x6A>(a1e, 0xFF0FFF0Fu, 0x00800080u), a2o = lop3<0x6A>(a1o, 0xFF0FFF0Fu, 0x00800080u);
+                    const uint32_t b2e = lop3<0x6A>(b1e, 0xFF0FFF0Fu, 0x00800080u), b2o = lop3<0x6A>(b1o, 0xFF0FFF0Fu, 0x00800080u);
+                    const uint32_t E0 = fma_f16x2(a1e, sA, cA), E1 = fma_f16x2(a2e, sA, cA);
+                    const uint32_t E2 = fma_f16x2(b1e, sB, cB), E3 = fma_f16x2(b2e, sB, cB);
+                    const uint32_t O0 = fma_f16x2(a1o, sA, cA), O1 = fma_f16x2(a2o, sA, cA);
+                    const uint32_t O2 = fma_f16x2(b1o, sB, cB), O3 = fma_f16x2(b2o, sB, cB);
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        mma_f16(o[nt][2 * x], E0, E1, E2, E3, pb[nt][0], pb[nt][1]);
+                        mma_f16(o[nt][2 * x + 1], O0, O1, O2, O3, pb[nt][0], pb[nt][1]);
+                    }
+                }
+            }
+        };
+
+        for (int it = 0; it < cr.n_tiles; ++it) {
+            if (!mbar_wait_bounded(bar0 + 8 * stage, parity)) { timed_out = true; break; }
+            const uint8_t* st = wsm + stage * G_::STAGE_BYTES;
+            const int n_live = cr.n_tok - it * kTile;        // tokens of this tile that exist (may exceed kTile)
+            if (n_live >= kTile) tile_body(st, n_live, std::true_type{});
+            else tile_body(st, n_live, std::false_type{});
+            __syncwarp();
+            issue_next(stage);
+            if (++stage == kStages) { stage = 0; parity ^= 1u; }
+        }
+        if (timed_out) break;
+
+        // ---- partial result of the run, at the slot of its first chunk ----------------------------
+        // row of kind 1 = 16*o_hi + o_lo, row of kind 2 = o_lo; common factor 2^(dv - 129 - kTopShift)
+        const float vfac = pow2_split(1.f, dv - 129 - kTopShift);
+        const float vfac16 = vfac * 0.0625f;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            float l = l_run[nt];
+            l += __shfl_xor_sync(0xffffffffu, l, 4);
+            l += __shfl_xor_sync(0xffffffffu, l, 8);
+            l += __shfl_xor_sync(0xffffffffu, l, 16);
+            const int qi = 4 * nt + t;
+            if (qi < Gq) {
+                float* dst = a.partials + (((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + qi) * a.n_chunks + cr.chunk0) * kPartStride;
+#pragma unroll
+                for (int r4 = 0; r4 < 4; ++r4) {
+                    const float w0 = o[nt][2 * r4][0] + o[nt][2 * r4][1], l0 = o[nt][2 * r4][2] + o[nt][2 * r4][3];
+                    const float w1 = o[nt][2 * r4 + 1][0] + o[nt][2 * r4 + 1][1], l1 = o[nt][2 * r4 + 1][2] + o[nt][2 * r4 + 1][3];
+                    float4 v;
+                    v.x = l0 * vfac;            // slot 16g + 4r4     (low nibble of byte 2r4)
+                    v.y = (w0 - l0) * vfac16;   // slot 16g + 4r4 + 1 (high nibble of byte 2r4)
+                    v.z = l1 * vfac;
+                    v.w = (w1 - l1) * vfac16;
+                    reinterpret_cast<float4*>(dst + 16 * g)[r4] = v;
+                }
+                if (g == 0) { dst[D] = m_run[nt]; dst[D + 1] = l; }
+            }
+        }
+    }
+
+    if (timed_out) {
+        // give the copies still in flight a bounded chance to land before the shared memory is released
+        if (lane == 0) raise_flag(a.status, KVBFP_FLAG_WAIT_TIMEOUT);
+        for (int s = 0; s < kStages; ++s) {
+            (void)mbar_wait_bounded(bar0 + 8 * s, 0);
+            (void)mbar_wait_bounded(bar0 + 8 * s, 1);
+        }
+    }
+}
+
+template <int N, int NT>
+kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
+    using G_ = Geo4<N>;
+    static int resident[64] = {0};          // thread blocks that fit the whole device, per device
+    int dev = 0;
+    KVBFP_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return KVBFP_ERR_UNSUPPORTED;
+    if (!resident[dev]) {
+        KVBFP_CUDA(cudaFuncSetAttribute(decode_mma4<N, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_::SMEM_BYTES));
+        int per_sm = 0, n_sm = 0;
+        KVBFP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_mma4<N, NT>, kWarps * 32, G_::SMEM_BYTES));
+        KVBFP_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+        if (per_sm < 1 || n_sm < 1) return KVBFP_ERR_CUDA;
+        resident[dev] = per_sm * n_sm;
+    }
+    // per-query exponents sit behind the fragments in the query region of the workspace
+    int32_t* qexp = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
+                                               (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
+    const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
+    make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qexp);
+    KVBFP_LAUNCH_CHECK("make_qfrag4");
+    const int64_t n_items = (int64_t)a.fmt.batch * a.fmt.n_kv_heads * a.n_chunks;
+    const int64_t want = (n_items + kWarps - 1) / kWarps;
+    const int grid = (int)(want < resident[dev] ? want : resident[dev]);
+    *n_warps = grid * kWarps;
+    cudaEvent_t ev0, ev1;
+    profile_events(&ev0, &ev1);
+    if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
+    decode_mma4<N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(a, qexp);
+    KVBFP_LAUNCH_CHECK("decode_mma4");
+    if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
+    return KVBFP_OK;
+}
+
+template <int N>
+kvbfp_status launch2(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
+    const int G = a.n_q_heads / a.fmt.n_kv_heads;
+    return (G <= 4) ? launch3<N, 1>(a, s, n_warps) : launch3<N, 2>(a, s, n_warps);
+}
+
+}  // namespace
+
+kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
+    switch (a.fmt.block) {
+        case 16: return launch2<16>(a, s, n_warps);
+        case 32: return launch2<32>(a, s, n_warps);
+        case 64: return launch2<64>(a, s, n_warps);
+        case 128: return launch2<128>(a, s, n_warps);
+    }
+    return KVBFP_ERR_UNSUPPORTED;
+}
+
+}  // namespace kvbfp

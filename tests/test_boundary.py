@@ -86,7 +86,7 @@ def test_host_side_argument_errors():
     assert L.kvbfp_decode_attn(*args(wsb=need - 1)) == B.ERR_WORKSPACE
     assert L.kvbfp_decode_attn(*args(ws=8)) == B.ERR_ALIGNMENT
     assert L.kvbfp_decode_attn(*args(qb=4)) == B.ERR_UNSUPPORTED
-    assert L.kvbfp_decode_attn(*args(flags=3)) == B.ERR_INVALID_ARG
+    assert L.kvbfp_decode_attn(*args(flags=4)) == B.ERR_INVALID_ARG
     assert L.kvbfp_decode_attn(*args(scale=-1.0)) == B.ERR_INVALID_ARG
     assert L.kvbfp_device_status(None, None) == B.ERR_INVALID_ARG
     assert B.launch_count() == before

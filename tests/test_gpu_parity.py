@@ -231,7 +231,7 @@ def run_decode_case(oracle, w, Bn, S, lens, block, p, impl, use_perm=True, perm_
     return host(out).astype(np.float64), ref
 
 
-IMPLS = [B.DECODE_SIMT, B.DECODE_MMA]
+IMPLS = [B.DECODE_SIMT, B.DECODE_MMA, B.DECODE_MMA_BF16]
 
 
 @pytest.mark.parametrize("impl", IMPLS)
