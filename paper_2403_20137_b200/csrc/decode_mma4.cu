@@ -52,7 +52,7 @@ namespace {
 #define KVBFP4_STAGES 2
 #endif
 #ifndef KVBFP4_MIN_CTAS
-#define KVBFP4_MIN_CTAS 1
+#define KVBFP4_MIN_CTAS 3
 #endif
 
 constexpr int kWarps = KVBFP4_WARPS;
