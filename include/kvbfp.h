@@ -27,7 +27,8 @@
  * Storage layout (the paper does not fix one; this is the library's own):
  *  - mantissa plane  [batch, n_kv_heads, max_seq, row_m] bytes, row_m = head_dim*p/8;
  *    a row is a little-endian bit stream, stored slot j in bits [j*p, (j+1)*p),
- *    two's complement (p = 4: low nibble is the even slot);
+ *    holding M + 2^(p-1) (excess code: 0 is stored as 8, 32 or 128; p = 4: low nibble is the even
+ *    slot);
  *  - exponent plane  [batch, n_kv_heads, max_seq, row_e] bytes, row_e = head_dim/n;
  *    byte i belongs to slots [i*n, (i+1)*n) and holds E + 127, where 2^E is the
  *    largest power of two not above the block's largest magnitude (E >= -127);

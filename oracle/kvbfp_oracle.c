@@ -82,7 +82,7 @@ void oracle_pack_mantissas(const int* M, int count, int p, uint8_t* bytes) {
     memset(bytes, 0, nbytes);
     const unsigned mask = (1u << p) - 1u;
     for (int j = 0; j < count; ++j) {
-        unsigned field = (unsigned)M[j] & mask;   /* two's complement, p bits */
+        unsigned field = (unsigned)(M[j] + (1 << (p - 1))) & mask;   /* excess-2^(p-1) code, p bits */
         for (int k = 0; k < p; ++k) {
             size_t bit = (size_t)j * (size_t)p + (size_t)k;
             if ((field >> k) & 1u) bytes[bit >> 3] |= (uint8_t)(1u << (bit & 7));
@@ -97,9 +97,7 @@ void oracle_unpack_mantissas(const uint8_t* bytes, int count, int p, int* M) {
             size_t bit = (size_t)j * (size_t)p + (size_t)k;
             field |= (unsigned)((bytes[bit >> 3] >> (bit & 7)) & 1u) << k;
         }
-        int v = (int)field;
-        if (field & (1u << (p - 1))) v -= (1 << p);   /* sign-extend */
-        M[j] = v;
+        M[j] = (int)field - (1 << (p - 1));   /* excess-2^(p-1) code */
     }
 }
 

@@ -64,7 +64,7 @@ double oracle_bfp_value(int M, int e8, int p);
 /* Cast one block of n doubles (Sec. II-B).  Writes the exponent byte and n mantissas. */
 int oracle_bfp_cast_block(const double* x, int n, int p, int* e8_out, int* M_out);
 
-/* p-bit two's-complement fields, element j in bits [j*p, (j+1)*p) of a
+/* p-bit fields holding M + 2^(p-1) (excess code), element j in bits [j*p, (j+1)*p) of a
  * little-endian bit stream. */
 void oracle_pack_mantissas(const int* M, int count, int p, uint8_t* bytes);
 void oracle_unpack_mantissas(const uint8_t* bytes, int count, int p, int* M);

@@ -121,12 +121,12 @@ __global__ void __launch_bounds__(kThreads) append_quant_pack(AppendArgs a) {
         if (P == 4) {
             uint32_t w = 0;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) w |= ((uint32_t)m[i] & 0xfu) << (4 * i);
+            for (int i = 0; i < 8; ++i) w |= ((uint32_t)(m[i] + 8) & 0xfu) << (4 * i);      // excess-8 code
             reinterpret_cast<uint32_t*>(mrow)[sub] = w;
         } else if (P == 6) {
             uint64_t w = 0;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) w |= ((uint64_t)((uint32_t)m[i] & 0x3fu)) << (6 * i);
+            for (int i = 0; i < 8; ++i) w |= ((uint64_t)((uint32_t)(m[i] + 32) & 0x3fu)) << (6 * i);     // excess-32 code
             uint16_t* o = reinterpret_cast<uint16_t*>(mrow + sub * 6);
             o[0] = (uint16_t)w;
             o[1] = (uint16_t)(w >> 16);
@@ -135,8 +135,8 @@ __global__ void __launch_bounds__(kThreads) append_quant_pack(AppendArgs a) {
             uint32_t lo = 0, hi = 0;
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                lo |= ((uint32_t)m[i] & 0xffu) << (8 * i);
-                hi |= ((uint32_t)m[i + 4] & 0xffu) << (8 * i);
+                lo |= ((uint32_t)(m[i] + 128) & 0xffu) << (8 * i);       // excess-128 code
+                hi |= ((uint32_t)(m[i + 4] + 128) & 0xffu) << (8 * i);
             }
             reinterpret_cast<uint2*>(mrow)[sub] = make_uint2(lo, hi);
         }

@@ -62,12 +62,11 @@ __device__ __forceinline__ float unit_weight(int e8, int p) {
 
 __device__ __forceinline__ void raise_flag(uint32_t* status, uint32_t bit) { atomicOr(status, bit); }
 
-// Sign-extended p-bit field starting at bit `bit` of a little-endian byte row.
+// Mantissa stored in the p-bit field (excess-2^(p-1) code) starting at bit `bit` of a little-endian byte row.
 __device__ __forceinline__ int extract_field(const uint8_t* row, int bit, int p) {
     int byte = bit >> 3, sh = bit & 7;
     uint32_t w = row[byte] | ((uint32_t)row[byte + ((sh + p > 8) ? 1 : 0)] << 8);
-    int v = (int)((w >> sh) & ((1u << p) - 1u));
-    return (v ^ (1 << (p - 1))) - (1 << (p - 1));
+    return (int)((w >> sh) & ((1u << p) - 1u)) - (1 << (p - 1));
 }
 
 }  // namespace kvbfp

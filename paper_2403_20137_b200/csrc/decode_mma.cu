@@ -8,7 +8,7 @@
 // them, an mbarrier per stage counts the bytes); there is no block-wide barrier in the loop.
 //
 // Arithmetic.  A mantissa field is turned into a bf16 number without an integer-to-float
-// conversion: the field (sign bit flipped, so it is an unsigned offset) is or-ed under the bits of
+// conversion: the stored field (an unsigned offset, M + 2^(P-1)) is or-ed under the bits of
 // 128.0, giving 128 + offset exactly; one bf16x2 fma with the block's power-of-two weight removes
 // the bias and applies 2^e in the same instruction, exactly (the result M * 2^e has at most 7
 // significant bits).  Scores:  S[16 tokens x 8 cols] += K[16 x 16 slots] . Q[16 slots x 8 cols],
@@ -61,12 +61,12 @@ __device__ __forceinline__ uint32_t weight_bf16(uint32_t e8) {
     return f >= 1 ? ((uint32_t)f << 7) : (0x40u >> (-f));
 }
 
-// Format constants of the "or under 128.0" conversion.  The field with its sign bit flipped is
-// M + 2^(P-1) (P = 4, 6); the value built is 128 + 2^(P-1) + M, so the bias to remove is `bias`.
+// Format constants of the "or under 128.0" conversion.  The stored field is M + 2^(P-1) (P = 4, 6);
+// the value built is 128 + 2^(P-1) + M, so the bias to remove is `bias`.
 template <int P> struct Fmt;
-template <> struct Fmt<4> { static constexpr uint32_t mask = 0x000F000Fu, magic = 0x43084308u, bias = 0xC308C308u; };  // -136
-template <> struct Fmt<6> { static constexpr uint32_t mask = 0x003F003Fu, magic = 0x43204320u, bias = 0xC320C320u; };  // -160
-template <> struct Fmt<8> { static constexpr uint32_t mask = 0x000F000Fu, magic = 0x43084308u, bias = 0xC510C510u; };  // -2304
+template <> struct Fmt<4> { static constexpr uint32_t mask = 0x000F000Fu, magic = 0x43004300u, bias = 0xC308C308u; };  // -136
+template <> struct Fmt<6> { static constexpr uint32_t mask = 0x003F003Fu, magic = 0x43004300u, bias = 0xC320C320u; };  // -160
+template <> struct Fmt<8> { static constexpr uint32_t mask = 0x000F000Fu, magic = 0x43004300u, bias = 0xC510C510u; };  // -2304
 
 // Per-row (or per token pair) weights ready for the conversion fma's.
 struct Wgt {
@@ -87,13 +87,13 @@ __device__ __forceinline__ Wgt make_wgt(uint32_t s2, uint32_t c2) {
 template <int P>
 __device__ __forceinline__ uint32_t cvt_pair(uint32_t x, const Wgt& w) {
     if (P == 8) {
-        // byte = 16*H + L, H signed high nibble, L unsigned low nibble
+        // byte = M + 128 = 16*H + L with both nibbles unsigned
         uint32_t lo = lop3<0xEA>(x, 0x000F000Fu, 0x43004300u);         // (x & m) | 128.0  = 128 + L
-        uint32_t hi = lop3<0x6A>(x >> 4, 0x000F000Fu, 0x43084308u);    // (x & m) ^ 136.0  = 136 + H
-        uint32_t v = fma_bf16x2(hi, w.s16, w.c);                       // (16H - 128) * 2^e, exact
-        return fma_bf16x2(lo, w.s, v);                                 // (16H + L) * 2^e, exact
+        uint32_t hi = lop3<0xEA>(x >> 4, 0x000F000Fu, 0x43004300u);    // (x & m) | 128.0  = 128 + H
+        uint32_t v = fma_bf16x2(hi, w.s16, w.c);                       // (16H - 256) * 2^e, exact
+        return fma_bf16x2(lo, w.s, v);                                 // (16H + L - 128) * 2^e = M * 2^e, exact
     }
-    return fma_bf16x2(lop3<0x6A>(x, Fmt<P>::mask, Fmt<P>::magic), w.s, w.c);   // (x & mask) ^ magic in one op
+    return fma_bf16x2(lop3<0xEA>(x, Fmt<P>::mask, Fmt<P>::magic), w.s, w.c);   // (x & mask) | 128.0 in one op
 }
 
 // Right shifts of a packed word by 4, 8 and 12; two of the three run on the multiply-add pipe.

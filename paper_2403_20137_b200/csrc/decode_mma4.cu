@@ -12,7 +12,7 @@
 // There is no block-wide barrier in the loop and no cluster multicast.
 //
 // Unpacking is what limits this kernel (integer-pipe instructions, not memory).  A packed byte holds
-// two mantissas; with the sign bits flipped it is B = 16*(M_hi+8) + (M_lo+8).  fp16 has a 10-bit
+// two mantissas in excess-8 code: B = 16*(M_hi+8) + (M_lo+8).  fp16 has a 10-bit
 // fraction, so the whole byte can be put under the bits of 1024.0 with one byte permute: the element
 // 1024 + B.  A second element with the high nibble masked away and bit 7 set, 1024 + 128 + (M_lo+8),
 // comes from one logic op.  One f16x2 fma per register with the block's power of two removes the
@@ -66,7 +66,6 @@ constexpr int kLutEntries = 512;        // index = exponent byte - D + 255, D = 
 
 constexpr uint32_t kMagic = 0x64646464u;        // 0x64 = high byte of fp16 1024.0
 constexpr uint32_t kBias = 0xE488E488u;         // fp16 -1160.0 twice
-constexpr uint32_t kFlip = 0x88888888u;         // flips the sign bit of every 4-bit field: M -> M + 8
 
 // fp16 bit pattern of 2^j for j in [-24, 15], 0 below.
 __device__ __forceinline__ uint32_t pow2_f16(int j) {
@@ -375,8 +374,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                 }
                 const uint4 xa = *reinterpret_cast<const uint4*>(st + k_off + mt * 16 * ROW_M);
                 const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off + (mt * 16 + 8) * ROW_M);
-                const uint32_t wa[4] = {xa.x ^ kFlip, xa.y ^ kFlip, xa.z ^ kFlip, xa.w ^ kFlip};      // sign bits -> offsets
-                const uint32_t wb[4] = {xb.x ^ kFlip, xb.y ^ kFlip, xb.z ^ kFlip, xb.w ^ kFlip};
+                const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wb[4] = {xb.x, xb.y, xb.z, xb.w};
                 uint2 la[NBK], lb[NBK];
 #pragma unroll
                 for (int k = 0; k < NBK; ++k) {
@@ -494,8 +492,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                     const uint32_t wA0 = (x < 2) ? vw[0].x : vw[0].y, wA1 = (x < 2) ? vw[1].x : vw[1].y;
                     const uint32_t wB0 = (x < 2) ? vw[2].x : vw[2].y, wB1 = (x < 2) ? vw[3].x : vw[3].y;
                     const uint32_t sel = (x & 1) ? 0x7632u : 0x5410u;
-                    // [tok.b, tok.b', tok'.b, tok'.b'] with the sign bits turned into offsets
-                    const uint32_t XA = prmt(wA0, wA1, sel) ^ kFlip, XB = prmt(wB0, wB1, sel) ^ kFlip;
+                    const uint32_t XA = prmt(wA0, wA1, sel), XB = prmt(wB0, wB1, sel);     // [tok.b, tok.b', tok'.b, tok'.b']
                     // kind 1 for the even byte by mask-or, for the odd byte by byte permute; kind 2 from kind 1
                     const uint32_t a1e = lop3<0xEA>(XA, 0x00FF00FFu, 0x64006400u), a1o = prmt(XA, kMagic, 0x4341u);
                     const uint32_t b1e = lop3<0xEA>(XB, 0x00FF00FFu, 0x64006400u), b1o = prmt(XB, kMagic, 0x4341u);

@@ -36,13 +36,12 @@ __device__ __forceinline__ void load_chunk(const uint8_t* p, uint32_t (&w)[P]) {
     }
 }
 
-// Slot i (compile-time) of a lane's 32-slot chunk, sign-extended.
+// Slot i (compile-time) of a lane's 32-slot chunk: the stored field is M + 2^(P-1).
 template <int P>
 __device__ __forceinline__ float slot_value(const uint32_t (&w)[P], int i) {
     const int bit = i * P, word = bit >> 5, sh = bit & 31;
     uint32_t v = (sh + P > 32) ? __funnelshift_r(w[word], w[(word + 1) % P], sh) : (w[word] >> sh);
-    int m = (int)(v << (32 - P)) >> (32 - P);
-    return (float)m;
+    return (float)((int)(v & ((1u << P) - 1u)) - (1 << (P - 1)));
 }
 
 template <int P, int N>

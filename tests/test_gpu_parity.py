@@ -114,7 +114,7 @@ def test_append_identity_and_single_plane(oracle):
     oc = oracle_cache(oracle, k, None, "bf16", 32, 4, 64)
     assert np.array_equal(host(gc.k_mant[0, :, :50]), oc.k_mant[0, :, :50])
     assert np.array_equal(host(gc.k_exp[0, :, :50]), oc.k_exp[0, :, :50])
-    assert not bool(gc.v_mant.any())          # V untouched
+    assert not bool(gc.v_mant.any())          # V untouched (the cache was created filled with zero bytes)
     B.append(gc, None, dev(v), dev(torch.zeros(1, dtype=torch.int32)))
     oc2 = oracle_cache(oracle, v, None, "bf16", 32, 4, 64)
     assert np.array_equal(host(gc.v_mant[0, :, :50]), oc2.k_mant[0, :, :50])

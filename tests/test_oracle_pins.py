@@ -133,20 +133,23 @@ def test_pack_all_values_all_positions(oracle, p):
             # independent writer: one Python integer as the little-endian bit stream
             stream = 0
             for j, m in enumerate(M):
-                stream |= (int(m) % (1 << p)) << (j * p)
+                stream |= ((int(m) + (1 << (p - 1))) % (1 << p)) << (j * p)     # excess code
             ref = np.frombuffer(stream.to_bytes(n * p // 8, "little"), dtype=np.uint8)
             assert np.array_equal(b, ref)
             assert np.array_equal(oracle.unpack_mantissas(b, n, p), M)
 
 
 def test_pack_nibble_and_six_bit_examples(oracle):
-    # p=4: low nibble = even element.  1 -> 0x1, -1 -> 0xF, 7 -> 0x7, -7 -> 0x9
-    assert list(oracle.pack_mantissas([1, -1, 7, -7], 4)) == [0xF1, 0x97]
-    # p=6: four elements in three bytes
-    assert list(oracle.pack_mantissas([1, 0, 0, 0], 6)) == [1, 0, 0]
-    assert list(oracle.pack_mantissas([0, 1, 0, 0], 6)) == [0x40, 0, 0]
-    assert list(oracle.pack_mantissas([0, 0, 1, 0], 6)) == [0, 0x10, 0]
-    assert list(oracle.pack_mantissas([0, 0, 0, -1], 6)) == [0, 0, 0xFC]
+    # p=4, excess-8 code, low nibble = even element.  1 -> 9, -1 -> 7, 7 -> 0xF, -7 -> 1, 0 -> 8
+    assert list(oracle.pack_mantissas([1, -1, 7, -7], 4)) == [0x79, 0x1F]
+    assert list(oracle.pack_mantissas([0, 0], 4)) == [0x88]
+    # p=6, excess-32 code: four elements in three bytes; all zero = fields 32 -> bits 100000 x4
+    z = int("100000" * 4, 2)
+    assert list(oracle.pack_mantissas([0, 0, 0, 0], 6)) == list(z.to_bytes(3, "little"))
+    assert list(oracle.pack_mantissas([1, 0, 0, 0], 6)) == list((z + 1).to_bytes(3, "little"))
+    assert list(oracle.pack_mantissas([0, 0, 0, -1], 6)) == list((z - (1 << 18)).to_bytes(3, "little"))
+    # p=8, excess-128 code
+    assert list(oracle.pack_mantissas([0, 127, -127], 8)) == [128, 255, 1]
 
 
 # ---------------------------------------------------------------- I9: argsort
@@ -223,12 +226,12 @@ def test_append_layout_and_positions(oracle):
     k[1, 1, 2, 17] = -3.0        # block 1
     oracle.append(c, k, None, "f32", np.array([4, 7], dtype=np.int32))
     row = c.k_mant[1, 2, 8]
-    assert row[0] == 0x04 and not row[1:8].any()            # M = 2^(p-2) = 4 in the low nibble
-    assert row[8] == 0xA0 and not row[9:].any()             # -3 -> t = -6 -> nibble 0xA, odd element
+    assert row[0] == 0x8C and (row[1:8] == 0x88).all()      # M = 2^(p-2) = 4 -> code 12 in the low nibble, zeros -> 8
+    assert row[8] == 0x28 and (row[9:] == 0x88).all()       # -3 -> t = -6 -> code 2, odd element
     assert list(c.k_exp[1, 2, 8]) == [127, 128]
-    assert (c.k_mant[1, 2, 7] == 0).all() and (c.k_exp[1, 2, 7] == 0).all()   # zero row written
+    assert (c.k_mant[1, 2, 7] == 0x88).all() and (c.k_exp[1, 2, 7] == 0).all()   # zero row written (code 8 = 0)
     assert (c.k_mant[1, 2, 6] == 0xAB).all() and (c.k_mant[0, 0, 3] == 0xAB).all()
-    assert (c.k_mant[0, 0, 4] == 0).all() and (c.k_mant[0, 0, 6] == 0xAB).all()
+    assert (c.k_mant[0, 0, 4] == 0x88).all() and (c.k_mant[0, 0, 6] == 0xAB).all()
     with pytest.raises(oracle.OracleError) as e:
         oracle.append(c, k, None, "f32", np.array([4, 9], dtype=np.int32))
     assert e.value.status == oracle.CAPACITY
@@ -269,7 +272,7 @@ def test_identity_permutation_is_plain_bfp(oracle):
 
 def test_dequant_matches_eq1_by_hand(oracle):
     c = oracle.Cache(1, 1, 16, 2, 8, 4)
-    c.k_mant[0, 0, 1] = np.frombuffer(bytes([0x21, 0x43, 0x65, 0x07, 0xFF, 0x9F, 0x00, 0x10]), dtype=np.uint8)
+    c.k_mant[0, 0, 1] = np.frombuffer(bytes([0xA9, 0xCB, 0xED, 0x8F, 0x77, 0x17, 0x88, 0x98]), dtype=np.uint8)
     c.k_exp[0, 0, 1] = [129, 120]
     out = oracle.dequant(c, "k", 0, 0, 1, 1)[0]
     want = [1, 2, 3, 4, 5, 6, 7, 0] + [m * 2.0 ** -9 for m in (-1, -1, -1, -7, 0, 0, 0, 1)]
