@@ -13,6 +13,8 @@ data-path collective (weak scaling); time is the max over ranks.
 Prints ONE JSON line on rank 0.
 """
 import argparse
+import dataclasses
+import hashlib
 import json
 import os
 import statistics
@@ -31,16 +33,42 @@ from paper_2403_20137_b200 import workloads as W  # noqa: E402
 METRIC = "decode_attn_tokens_per_s"
 UNIT = "tokens/s"
 
+# DRAM traffic of the dominant kernel from one ncu capture (profiles/decode_mma4_b4_s8192_ncu_full.md):
+# dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
+# same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
+# value recorded with the capture; otherwise the bench reports null.
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": None, "sources_sha256": None}}
+KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
+
+
+def sources_hash(kernel):
+    h = hashlib.sha256()
+    for rel in KERNEL_SOURCES.get(kernel, []):
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def traffic_per_launch(kernel, units):
+    t = TRAFFIC.get(kernel)
+    if not t or not t["bytes_per_unit"] or t["sources_sha256"] != sources_hash(kernel):
+        return None
+    return t["bytes_per_unit"] * units
+
 
 def workload_name(w):
     return (f"config{w.config}: B{w.batch} Hq{w.n_q_heads} Hkv{w.n_kv_heads} d{w.head_dim} S{w.seq} {w.dtype} "
             f"BFP block{w.block} mant{w.mant_bits}; append 1 token/seq + decode attention")
 
 
+def decode_units(w):
+    return w.batch * w.n_kv_heads * w.seq
+
+
 def decode_bytes(w):
     """Algorithmic bytes of one decode launch: packed K and V rows of every cached token, once."""
     row = w.head_dim * w.mant_bits // 8 + w.head_dim // w.block
-    return 2 * row * w.batch * w.n_kv_heads * w.seq
+    return 2 * row * decode_units(w)
 
 
 def measured_peak():
@@ -50,6 +78,20 @@ def measured_peak():
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs, copy bandwidth)"
     except Exception:
         return 6650.0, "fallback (6.65 TB/s, earlier copy measurement on this pool)"
+
+
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_throughput(per_rank_units, world, ms_per_step_max):
+    """Units all ranks processed per second, timed by the slowest rank."""
+    return world * per_rank_units / (ms_per_step_max * 1e-3)
 
 
 class ClockSampler:
@@ -168,6 +210,18 @@ def run_reference(args, w, rank):
     }))
 
 
+def timed(fn, reps=1):
+    """Milliseconds per call of fn(), CUDA events on the current stream."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -175,9 +229,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=3, choices=[2, 3, 4])
-    ap.add_argument("--decode-impl", default="auto", choices=["auto", "simt", "mma"])
+    ap.add_argument("--decode-impl", default="auto", choices=["auto", "simt", "mma", "mma_bf16"])
     ap.add_argument("--ref-units", type=int, default=0, help="(batch, kv head) units per step of the reference arm (0 = sized for ~100 s)")
-    ap.add_argument("--cpu-baseline-units", type=int, default=256)
+    ap.add_argument("--cpu-baseline-units", type=int, default=512)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small cases for profiling)")
     ap.add_argument("--seq", type=int, default=0, help="override the cached sequence length")
@@ -185,9 +239,9 @@ def main():
     ap.add_argument("--block", type=int, default=0, choices=[0, 16, 32, 64, 128])
     ap.add_argument("--chunk", type=int, default=0, help="tokens per sequence chunk (0 = library default)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the set-up timings and the quality report")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
-    import dataclasses
     over = {k: v for k, v in (("batch", args.batch), ("seq", args.seq), ("mant_bits", args.mant_bits),
                               ("block", args.block)) if v}
     if over:
@@ -211,18 +265,51 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    # ---- set-up (untimed): calibrate, prefill S-1 tokens -----------------------------------------
-    impl = {"auto": B.DECODE_AUTO, "simt": B.DECODE_SIMT, "mma": B.DECODE_MMA}[args.decode_impl]
+    # ---- set-up (untimed for the step metric): calibrate, prefill S-1 tokens ----------------------
+    impl = {"auto": B.DECODE_AUTO, "simt": B.DECODE_SIMT, "mma": B.DECODE_MMA, "mma_bf16": B.DECODE_MMA_BF16}[args.decode_impl]
+    kernel = "decode_simt" if impl == B.DECODE_SIMT else \
+        ("decode_mma4" if (w.mant_bits == 4 and impl != B.DECODE_MMA_BF16) else "decode_mma")
     S, Bn, Hkv, Hq, d = w.seq, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim
+    es = 2 if w.dtype == "bf16" else 4
+    extras = {}
     calib = W.make_calibration(w, device=dev)
     _, perm_k, _ = B.calibrate(calib, Hkv, d)
+    if not args.no_extras:
+        ms = timed(lambda: B.calibrate(calib, Hkv, d), reps=3)
+        extras["calibrate"] = {"tokens": int(calib.shape[0]), "ms": ms, "GB/s": calib.numel() * es / ms / 1e6}
     del calib
     cache = B.Cache(Bn, Hkv, d, S, w.block, w.mant_bits, device=dev)
     zeros = torch.zeros(Bn, dtype=torch.int32, device=dev)
     k, v = W.make_kv(w, n_tokens=S, device=dev)                      # [B, S, Hkv, d]
-    B.append(cache, k[:, :S - 1].contiguous(), v[:, :S - 1].contiguous(), zeros, perm_k=perm_k)
+    k_pre, v_pre = k[:, :S - 1].contiguous(), v[:, :S - 1].contiguous()
+    B.append(cache, k_pre, v_pre, zeros, perm_k=perm_k)
+    if not args.no_extras:
+        ms = timed(lambda: B.append(cache, k_pre, v_pre, zeros, perm_k=perm_k), reps=3)
+        rows = 2 * Bn * (S - 1) * Hkv
+        row_bytes = d * es + d * w.mant_bits // 8 + d // w.block
+        extras["append_prefill"] = {"tokens_per_seq": S - 1, "ms": ms, "GB/s": rows * row_bytes / ms / 1e6,
+                                    "elements/s": rows * d / (ms * 1e-3)}
+        # quality on one head: key MSE and pre-softmax score error with and without K-sort (Table I's direction)
+        Tq = max(16, min(4096, (S - 1) // 16 * 16))
+        plain = B.Cache(1, Hkv, d, Tq, w.block, w.mant_bits, device=dev)
+        sortd = B.Cache(1, Hkv, d, Tq, w.block, w.mant_bits, device=dev)
+        z1 = torch.zeros(1, dtype=torch.int32, device=dev)
+        kk = k[:1, :Tq].contiguous()
+        B.append(plain, kk, None, z1)
+        B.append(sortd, kk, None, z1, perm_k=perm_k)
+        ref = kk[0, :, 0].float()
+        dq_p = B.dequant(plain, "k", 0, 0, 0, Tq)
+        dq_s = B.dequant(sortd, "k", 0, 0, 0, Tq, perm=perm_k)
+        qv = W.make_q(w, device=dev)[0, 0].float()
+        s_ref = ref @ qv
+        extras["quality_head0"] = {
+            "bits_per_element": w.mant_bits + 8.0 / w.block,
+            "key_mse_unsorted": float(((dq_p - ref) ** 2).mean()), "key_mse_ksort": float(((dq_s - ref) ** 2).mean()),
+            "score_rms_err_unsorted": float(((dq_p @ qv - s_ref) ** 2).mean().sqrt()),
+            "score_rms_err_ksort": float(((dq_s @ qv - s_ref) ** 2).mean().sqrt())}
+        del plain, sortd, kk, dq_p, dq_s
     k_new, v_new = k[:, S - 1:].contiguous(), v[:, S - 1:].contiguous()
-    del k, v
+    del k, v, k_pre, v_pre
     q = W.make_q(w, device=dev)
     start_pos = torch.full((Bn,), S - 1, dtype=torch.int32, device=dev)
     seq_lens = torch.full((Bn,), S, dtype=torch.int32, device=dev)
@@ -290,48 +377,48 @@ def main():
     e2e_ok = bool(torch.equal(hout.to(dev), out)) if n_e2e else None
 
     # ---- max over ranks -----------------------------------------------------------------------------
-    if dist is not None:
-        t = torch.tensor([ms_total, ms_e2e, kernel_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e, kernel_ms = t.tolist()
+    ms_total, ms_e2e, kernel_ms = max_over_ranks([ms_total, ms_e2e, kernel_ms], dist, dev)
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
     ms_step = ms_total / args.steps
-    value = world * Bn / (ms_step * 1e-3)
-    e2e_value = world * Bn / (ms_e2e / args.steps * 1e-3)
+    value = whole_job_throughput(Bn, world, ms_step)
+    e2e_value = whole_job_throughput(Bn, world, ms_e2e / args.steps) if n_e2e else None
     peak, peak_src = measured_peak()
     alg = decode_bytes(w)
     achieved = alg / (kernel_ms * 1e-3) / 1e9
-    es = 2 if w.dtype == "bf16" else 4
     h2d = 2 * Bn * Hkv * d * es + Bn * Hq * d * es
     d2h = Bn * Hq * d * 4
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload_name(w), "per_gpu_batch": Bn, "decode_kernel": args.decode_impl,
+        "dtype": "f16" if kernel == "decode_mma4" else ("bf16" if kernel == "decode_mma" else "f32"),
+        "data": "synthetic",
+        "config": {"workload": workload_name(w), "per_gpu_batch": Bn, "decode_kernel": kernel,
                    "l2": f"inputs larger than L2: {alg / 1e6:.0f} MB of cache read per step vs 126 MB L2",
                    "device_status_flags": flags, "e2e_matches_device_path": e2e_ok},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": ms_e2e / args.steps},
+                "ms_per_step": (ms_e2e / args.steps) if n_e2e else None},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "decode_mma" if impl != B.DECODE_SIMT else "decode_simt",
-                     "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None, "algorithmic_bytes": alg, "kernel_ms": kernel_ms, "peak_source": peak_src},
+        "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "traffic": traffic_per_launch(kernel, decode_units(w)),
+                     "algorithmic_bytes": alg, "kernel_ms": kernel_ms, "peak_source": peak_src},
+        "extras": extras or None,
     }
     if not args.no_cpu_baseline and world == 1:
         sample = min(args.cpu_baseline_units, Bn * Hkv)
         ost = OracleStep(w, sample)
-        t, cores = ost.run(), ost.cores
+        reps = 2
+        t = statistics.mean(ost.run() for _ in range(reps))
         t_full = t * (Bn * Hkv) / sample
         result["cpu_baseline"] = {
-            "value": Bn / t_full, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"{sample} of {Bn * Hkv} (batch, kv head) units of one step, {t:.1f} s, scaled to the full step"}
+            "value": Bn / t_full, "unit": UNIT, "cores": ost.cores, "kind": "oracle",
+            "sample": (f"{sample} of {Bn * Hkv} (batch, kv head) units of one step, {reps} repetitions of {t:.2f} s on "
+                       f"{ost.cores} threads, scaled to the full step")}
     else:
         result["cpu_baseline"] = None
     print(json.dumps(result))

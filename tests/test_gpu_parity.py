@@ -337,3 +337,52 @@ def test_ksort_improves_gpu_cache_quality(oracle):
         mse_p += float(((B.dequant(plain, "k", 0, h, 0, 512) - ref) ** 2).mean())
         mse_s += float(((B.dequant(sortd, "k", 0, h, 0, 512, perm=perm) - ref) ** 2).mean())
     assert mse_s < 0.85 * mse_p
+
+
+# ------------------------------------------------------------------------------- full-size workloads
+def _full_size_case(oracle, cfg, sample_pairs):
+    """The benchmark's own launch (full batch, full sequence, library-chosen chunking) with inputs drawn on
+    the GPU; the oracle recomputes sampled (batch, kv head) units one by one from the same raw inputs."""
+    w = W.CONFIGS[cfg]
+    S, Bn, Hkv, Hq, d = w.seq, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim
+    G = Hq // Hkv
+    dv = torch.device("cuda")
+    calib = W.make_calibration(w, device=dv)
+    _, perm, _ = B.calibrate(calib, Hkv, d)
+    del calib
+    k, v = W.make_kv(w, n_tokens=S, device=dv)
+    q = W.make_q(w, device=dv)
+    cache = B.Cache(Bn, Hkv, d, S, w.block, w.mant_bits, device=dv)
+    zeros = torch.zeros(Bn, dtype=torch.int32, device=dv)
+    B.append(cache, k[:, :S - 1].contiguous(), v[:, :S - 1].contiguous(), zeros, perm_k=perm)
+    B.append(cache, k[:, S - 1:].contiguous(), v[:, S - 1:].contiguous(),
+             torch.full((Bn,), S - 1, dtype=torch.int32, device=dv), perm_k=perm)
+    lens = torch.full((Bn,), S, dtype=torch.int32, device=dv)
+    out = B.decode_attn(cache, q, lens, perm_k=perm, max_len_hint=S)
+    assert B.device_status() == 0
+    perm_h = host(perm)
+    worst = 0.0
+    for (b, h) in sample_pairs:
+        kk = W.to_oracle(k[b:b + 1, :, h:h + 1])
+        vv = W.to_oracle(v[b:b + 1, :, h:h + 1])
+        oc = oracle.Cache(1, 1, d, S, w.block, w.mant_bits)
+        oracle.append(oc, kk, vv, w.dtype, np.zeros(1, np.int32), perm_k=perm_h[h:h + 1])
+        # packed planes of the sampled unit are bit-exact at full size too
+        assert np.array_equal(host(cache.k_mant[b, h]), oc.k_mant[0, 0])
+        assert np.array_equal(host(cache.v_exp[b, h]), oc.v_exp[0, 0])
+        qq = W.to_oracle(q[b:b + 1, h * G:(h + 1) * G])
+        ref = oracle.decode_attn(oc, qq, w.dtype, G, [S], perm_k=perm_h[h:h + 1])
+        got = host(out[b:b + 1, h * G:(h + 1) * G]).astype(np.float64)
+        worst = max(worst, rel_err(got, ref))
+    assert worst <= ATTN_TOL
+    return worst
+
+
+def test_full_size_config3_sampled(oracle):
+    """B16, H32, S8192 (the benchmark workload): four sampled (batch, head) units."""
+    _full_size_case(oracle, 3, [(0, 0), (5, 17), (15, 31), (9, 3)])
+
+
+def test_full_size_config4_gqa_sampled(oracle):
+    """B8, 32 query heads on 8 KV heads, S32768: two sampled (batch, kv head) units, four query heads each."""
+    _full_size_case(oracle, 4, [(0, 0), (7, 5)])
