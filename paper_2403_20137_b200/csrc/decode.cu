@@ -76,7 +76,7 @@ size_t qfrag_bytes(const kvbfp_format& f, int n_q_heads) {
     const int group = n_q_heads / f.n_kv_heads;
     const int nt = (group + 3) / 4;                  // four query heads per 8-column MMA tile
     const size_t frag = (size_t)f.batch * f.n_kv_heads * nt * 8 * 32 * 2 * sizeof(uint32_t);
-    const size_t qexp = ((size_t)f.batch * n_q_heads * sizeof(int32_t) + 255) & ~(size_t)255;   // per-query exponents
+    const size_t qexp = ((size_t)f.batch * n_q_heads * 8 * sizeof(int32_t) + 255) & ~(size_t)255;   // per-query exponents and biases
     return frag + qexp;
 }
 

@@ -24,6 +24,15 @@
 //   output:  the row of kind 1 accumulates 16*o_hi + o_lo and the row of kind 2 accumulates o_lo;
 //            o_hi = (row1 - row2)/16 once, when the run's partial result is written.
 //
+// Scores for blocks of 32 slots or more use the integer tensor-core path instead (Sec. II-B of the paper:
+// the inner product of two BFP blocks is an integer product plus an exponent addition).  The packed
+// bytes are fed to an unsigned-byte x signed-byte MMA as they are (kind 1) and with the low nibble moved
+// up (kind 2 = 16 x low nibble): two integer ops per packed word and no conversion at all.  The query coefficients of
+// each block are cast to 15-bit fixed point with the block's own exponent and split into two signed
+// byte digits, which sit in two MMA columns; the two 32-bit sums of a (token, block) are recombined
+// exactly, the constant contribution of the offsets (136 per kind-1 byte, 128 per kind-2 byte) was put
+// into the accumulator beforehand, and one fp32 multiply-add applies 2^(e_k + e_q) per (token, block).
+//
 // Range.  fp16 cannot hold 2^e for every exponent byte, so each run first takes the largest K and V
 // exponent byte of its rows (D_k, D_v) and uses the weights 2^(e - D + 5): the largest block gets
 // 2^5 (the bias product 1160 * 2^5 still fits fp16), blocks more than 2^29 below the largest one of
@@ -88,7 +97,7 @@ __device__ __forceinline__ float pow2_split(float x, int ex) {
 // One warp per (batch, kv head, n-tile).  Writes, in MMA B-fragment order, the (hi, lo) fp16 halves of
 // the coefficients c1 = q_hi/16 (whole byte) and c2 = q_lo - q_hi/16 (low nibble), normalised per query
 // head by a power of two 2^qe, and qe itself.
-__global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t* qexp) {
+__global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t* qmeta) {
     const int N = a.fmt.block;
     const int lane = threadIdx.x, gp = lane >> 2, tp = lane & 3;
     const int item = blockIdx.x;
@@ -144,7 +153,7 @@ __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t*
         if (lane == 0) sqe[qq] = qe;
     }
     __syncwarp();
-    if (lane < 4 && 4 * nt + lane < G) qexp[(int64_t)b * a.n_q_heads + hk * G + 4 * nt + lane] = sqe[lane];
+    if (lane < 4 && 4 * nt + lane < G) qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + lane) * 8] = sqe[lane];
 
     const int qi = 4 * nt + (gp >> 1), part = gp & 1;
     uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32 * 2);
@@ -171,6 +180,99 @@ __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t*
     }
 }
 
+// Integer variant (blocks of 32 slots or more).  One warp per (batch, kv head, n-tile).  The coefficients of
+// every block are cast to C = round(c * 2^(14 - qe)) with the block's own exponent qe and written as two signed
+// byte digits, C = 256 * d1 + d0, in the B-fragment order of the byte MMA: fragment m = 2 * seg + kind covers the
+// bytes [16 seg, 16 seg + 16) of a row; lane (g, t) holds bytes 4t..4t+3 for column g = (query g/2, digit g%2:
+// 0 = d1, 1 = d0).  qmeta[query][2 blk] = qe, qmeta[query][2 blk + 1] = 136 * sum(C of kind 1) + 128 * sum(C of kind 2).
+__global__ void __launch_bounds__(32) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
+    const int N = a.fmt.block;
+    const int lane = threadIdx.x, gp = lane >> 2, tp = lane & 3;
+    const int item = blockIdx.x;
+    const int nt = item % NT, hk = (item / NT) % a.fmt.n_kv_heads, b = item / NT / a.fmt.n_kv_heads;
+    const int G = a.n_q_heads / a.fmt.n_kv_heads;
+    __shared__ float sq[4][D];       // pi(q) of the four query heads of this n-tile, then the coefficients
+    __shared__ int sC[4][D];         // fixed-point coefficients
+    for (int i = lane; i < 4 * D; i += 32) {
+        const int qq = 4 * nt + i / D, slot = i % D;
+        float v = 0.f;
+        if (qq < G) {
+            const int ch = a.perm_k ? (a.perm_k[hk * D + slot] & (D - 1)) : slot;
+            const int64_t idx = ((int64_t)b * a.n_q_heads + hk * G + qq) * D + ch;
+            v = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
+        }
+        sq[i / D][slot] = v;
+    }
+    __syncwarp();
+    const int nblk = D / N;
+    if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
+        for (int i = lane; i < 4 * nblk; i += 32) {
+            float* blk = &sq[i / nblk][(i % nblk) * N];
+            uint32_t am = 0;
+            for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(blk[j]) & 0x7fffffffu);
+            int e8 = (int)(am >> 23);
+            if (e8 == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e8 = 254; }
+            const int k = 127 - e8 + 6, k1 = k >> 1, k2 = k - k1;
+            const float w = unit_weight(e8, 8);
+            for (int j = 0; j < N; ++j) {
+                float tv = (blk[j] * pow2i(k1)) * pow2i(k2);
+                blk[j] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * w;
+            }
+        }
+        __syncwarp();
+    }
+    // coefficients in place: slot 2j+1 <- c1 = q_hi/16 (kind 1: whole byte), slot 2j <- c2 = (q_lo - q_hi/16)/16
+    // (kind 2: 16 x low nibble).  Both multiply operands that carry a factor 16, so they have the same size and
+    // one block exponent serves both without losing bits of either.
+    for (int i = lane; i < 4 * (D / 2); i += 32) {
+        float* pr2 = &sq[i / (D / 2)][2 * (i % (D / 2))];
+        const float c1 = pr2[1] * 0.0625f, c2 = (pr2[0] - c1) * 0.0625f;
+        pr2[0] = c2;
+        pr2[1] = c1;
+    }
+    __syncwarp();
+    // per (query, block): exponent, fixed-point cast, bias
+    for (int i = lane; i < 4 * nblk; i += 32) {
+        const int qq = i / nblk, blk = i % nblk;
+        const float* c = &sq[qq][blk * N];
+        uint32_t am = 0;
+        for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(c[j]) & 0x7fffffffu);
+        int e = (int)(am >> 23);
+        if (e == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e = 254; }
+        const int qe = (am == 0) ? 0 : e - 126;               // |c| * 2^-qe < 1
+        const int sh = 14 - qe, h1 = sh / 2, h2 = sh - h1;    // two exact factors (sh in [-114, 140])
+        const float f1 = pow2i(h1), f2 = pow2i(h2);
+        int bias = 0;
+        for (int j = 0; j < N; ++j) {
+            const int C = __float2int_rn((c[j] * f1) * f2);
+            sC[qq][blk * N + j] = C;
+            bias += ((j & 1) ? 136 : 128) * C;
+        }
+        if (4 * nt + qq < G) {
+            int32_t* m = qmeta + ((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8;
+            m[2 * blk] = qe;
+            m[2 * blk + 1] = bias;
+        }
+    }
+    __syncwarp();
+    const int qq = gp >> 1, digit = gp & 1, qi = 4 * nt + qq;
+    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+        const int seg = m >> 1, kind = m & 1;
+        uint32_t reg = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int byte = 16 * seg + 4 * tp + e;
+            const int C = sC[qq][2 * byte + (kind == 0 ? 1 : 0)];
+            const int d1 = (C + 128) >> 8, d0 = C - 256 * d1;
+            const int dsel = (qi < G) ? (digit ? d0 : d1) : 0;
+            reg |= ((uint32_t)dsel & 0xffu) << (8 * e);
+        }
+        dst[((m >> 2) * 32 + lane) * 4 + (m & 3)] = reg;
+    }
+}
+
 // ------------------------------------------------------------------ main kernel
 template <int N>
 struct Geo4 {
@@ -182,7 +284,8 @@ struct Geo4 {
     static constexpr int STAGE_BYTES = 2 * kTile * (ROW_M + ROW_E);
     static constexpr int WARP_BYTES = kStages * STAGE_BYTES;
     static constexpr int LUT_OFF = kWarps * WARP_BYTES;                 // uint2[kLutEntries]
-    static constexpr int BAR_OFF = LUT_OFF + kLutEntries * 8;
+    static constexpr int LUTF_OFF = LUT_OFF + kLutEntries * 8;          // float[256] (integer score path)
+    static constexpr int BAR_OFF = LUTF_OFF + (N >= 32 ? 256 * 4 : 0);
     static constexpr int SMEM_BYTES = BAR_OFF + kWarps * kStages * 8;
 };
 
@@ -224,10 +327,12 @@ struct Run {
 };
 
 template <int N, int NT>
-__global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(DecodeArgs a, const int32_t* __restrict__ qexp) {
+__global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta) {
     using G_ = Geo4<N>;
     constexpr int ROW_E = G_::ROW_E;
     constexpr int NBK = (N == 16) ? 2 : 1;            // blocks inside a K lane chunk of 32 slots
+    constexpr bool KI = (N >= 32);                    // integer MMA path for the scores
+    constexpr int NBLK = KI ? D / N : 1;              // blocks of a row (integer path)
     extern __shared__ __align__(128) uint8_t smem[];
 
     // weight table: entry i = (2^(i - 255 + kTopShift) twice as f16x2, the same times -1160); entries
@@ -237,6 +342,10 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
         const uint32_t s2 = (i <= 255 ? pow2_f16(i - 255 + kTopShift) : 0u) * 0x00010001u;
         lut[i] = make_uint2(s2, mul_f16x2(s2, kBias));
     }
+    // integer score path: 2^(e - 129), the true weight of a mantissa unit, as fp32 (no range issue there)
+    float* lutf = reinterpret_cast<float*>(smem + G_::LUTF_OFF);
+    if (KI)
+        for (int i = threadIdx.x; i < 256; i += kWarps * 32) lutf[i] = unit_weight(i, 4);
     __syncthreads();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
@@ -311,7 +420,8 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
     for (int s = 0; s < kStages; ++s) issue_next(s);
 
     // per-lane byte offsets inside a stage
-    const int k_off = G_::KM_OFF + g * ROW_M + t * 16;
+    const int k_off = G_::KM_OFF + g * ROW_M + t * (KI ? 4 : 16);
+    const int kei_off = G_::KE_OFF + g * ROW_E;
     const int ke_off = G_::KE_OFF + g * ROW_E + ((N == 16) ? 2 * t : (N == 32) ? t : (N == 64) ? (t >> 1) : 0);
     const int v_off = G_::VM_OFF + t * ROW_M + g * 8;
     const int ve_off = G_::VE_OFF + t * ROW_E + (16 * g) / N;
@@ -328,25 +438,43 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
         if (cr.n_tok == 0) continue;
 
         // ---- run set-up: exponent references, query fragments, score factors ------------------
-        const int dk = warp_max_byte(a.k_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
+        const int dk = KI ? 0 : warp_max_byte(a.k_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
         const int dv = warp_max_byte(a.v_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
         const uint2* lutk = lut + (255 - dk);
         const uint2* lutv = lut + (255 - dv);
-        uint2 qf[NT][8];
+        uint2 qf[NT][8];                  // fp16 path: B fragments of the coefficients
         float kfac[NT];
+        uint32_t qi8[NT][8];              // integer path: B fragments of the coefficient digits
+        float qfac[NT][NBLK];             //   scale * log2(e) * 2^(qe - 14) per block
+        int qbias[NT][NBLK];              //   offset contribution per block
         {
-            const uint4* src = reinterpret_cast<const uint4*>(a.qfrag) + (((int64_t)cr.b * Hkv + cr.hk) * NT) * (4 * 32);
+            const uint4* src = reinterpret_cast<const uint4*>(a.qfrag);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
+                const int qn = 4 * nt + t;
+                const int32_t* meta = qmeta + ((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + (qn < Gq ? qn : 0)) * 8;
+                if (KI) {
+                    const uint4* s8 = src + (((int64_t)cr.b * Hkv + cr.hk) * NT + nt) * (2 * 32);
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 v = __ldg(src + (nt * 4 + j) * 32 + lane);
-                    qf[nt][2 * j] = make_uint2(v.x, v.y);
-                    qf[nt][2 * j + 1] = make_uint2(v.z, v.w);
+                    for (int j = 0; j < 2; ++j) {
+                        const uint4 v = __ldg(s8 + j * 32 + lane);
+                        qi8[nt][4 * j] = v.x; qi8[nt][4 * j + 1] = v.y; qi8[nt][4 * j + 2] = v.z; qi8[nt][4 * j + 3] = v.w;
+                    }
+#pragma unroll
+                    for (int k = 0; k < NBLK; ++k) {
+                        qfac[nt][k] = pow2_split(a.scale_log2e, meta[2 * k] - 14);
+                        qbias[nt][k] = meta[2 * k + 1];
+                    }
+                } else {
+                    const uint4* s16 = src + (((int64_t)cr.b * Hkv + cr.hk) * NT + nt) * (4 * 32);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint4 v = __ldg(s16 + j * 32 + lane);
+                        qf[nt][2 * j] = make_uint2(v.x, v.y);
+                        qf[nt][2 * j + 1] = make_uint2(v.z, v.w);
+                    }
+                    kfac[nt] = pow2_split(a.scale_log2e, dk - 129 - kTopShift + (qn < Gq ? meta[0] : 0));
                 }
-                const int qi = 4 * nt + t;
-                const int qe = (qi < Gq) ? qexp[(int64_t)cr.b * a.n_q_heads + cr.hk * Gq + qi] : 0;
-                kfac[nt] = pow2_split(a.scale_log2e, dk - 129 - kTopShift + qe);
             }
         }
         float o[NT][8][4];
@@ -372,44 +500,87 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                     for (int nt = 0; nt < NT; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = -INFINITY;
                     continue;
                 }
-                const uint4 xa = *reinterpret_cast<const uint4*>(st + k_off + mt * 16 * ROW_M);
-                const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off + (mt * 16 + 8) * ROW_M);
-                const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wb[4] = {xb.x, xb.y, xb.z, xb.w};
-                uint2 la[NBK], lb[NBK];
+                if (KI) {
+                    // ---- integer path: bytes as they are (kind 1) and 16 x low nibble (kind 2), per 16-byte segment
+                    int acc[NT][NBLK][4];
 #pragma unroll
-                for (int k = 0; k < NBK; ++k) {
-                    la[k] = lutk[st[ke_off + mt * 16 * ROW_E + k]];
-                    lb[k] = lutk[st[ke_off + (mt * 16 + 8) * ROW_E + k]];
-                }
-                float acc[NT][2][4];
+                    for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int kb = (NBK == 2) ? (i >> 1) : 0;
-                    // bytes 4i..4i+3 of the lane chunk: kind 1 by byte permute, kind 2 by one logic op
-                    const uint32_t a1_01 = prmt(wa[i], kMagic, 0x4140u), a1_23 = prmt(wa[i], kMagic, 0x4342u);
-                    const uint32_t b1_01 = prmt(wb[i], kMagic, 0x4140u), b1_23 = prmt(wb[i], kMagic, 0x4342u);
-                    const uint32_t a2_01 = lop3<0x6A>(a1_01, 0xFF0FFF0Fu, 0x00800080u), a2_23 = lop3<0x6A>(a1_23, 0xFF0FFF0Fu, 0x00800080u);
-                    const uint32_t b2_01 = lop3<0x6A>(b1_01, 0xFF0FFF0Fu, 0x00800080u), b2_23 = lop3<0x6A>(b1_23, 0xFF0FFF0Fu, 0x00800080u);
-                    const uint32_t A0 = fma_f16x2(a1_01, la[kb].x, la[kb].y), A1 = fma_f16x2(b1_01, lb[kb].x, lb[kb].y);
-                    const uint32_t A2 = fma_f16x2(a2_01, la[kb].x, la[kb].y), A3 = fma_f16x2(b2_01, lb[kb].x, lb[kb].y);
-                    const uint32_t B0 = fma_f16x2(a1_23, la[kb].x, la[kb].y), B1 = fma_f16x2(b1_23, lb[kb].x, lb[kb].y);
-                    const uint32_t B2 = fma_f16x2(a2_23, la[kb].x, la[kb].y), B3 = fma_f16x2(b2_23, lb[kb].x, lb[kb].y);
+                        for (int k = 0; k < NBLK; ++k) {      // the offsets' constant contribution goes in up front
+                            acc[nt][k][0] = 0; acc[nt][k][1] = -qbias[nt][k];
+                            acc[nt][k][2] = 0; acc[nt][k][3] = -qbias[nt][k];
+                        }
+                    const uint8_t* pa = st + k_off + mt * 16 * ROW_M;
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        const uint2 q0 = qf[nt][2 * i], q1 = qf[nt][2 * i + 1];
-                        if (i == 0) {
-                            mma_f16_first(acc[nt][0], A0, A1, A2, A3, q0.x, q0.y);
-                            mma_f16_first(acc[nt][1], B0, B1, B2, B3, q1.x, q1.y);
-                        } else {
-                            mma_f16(acc[nt][0], A0, A1, A2, A3, q0.x, q0.y);
-                            mma_f16(acc[nt][1], B0, B1, B2, B3, q1.x, q1.y);
+                    for (int seg = 0; seg < 4; ++seg) {
+                        const uint32_t wa = *reinterpret_cast<const uint32_t*>(pa + 16 * seg);
+                        const uint32_t wb = *reinterpret_cast<const uint32_t*>(pa + 8 * ROW_M + 16 * seg);
+                        const uint32_t la = (wa << 4) & 0xF0F0F0F0u, lb = (wb << 4) & 0xF0F0F0F0u;    // 16 x low nibble
+                        constexpr int SEG_PER_BLK = 4 / NBLK;
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            mma_u8s8(acc[nt][seg / SEG_PER_BLK], wa, wb, qi8[nt][2 * seg]);
+                            mma_u8s8(acc[nt][seg / SEG_PER_BLK], la, lb, qi8[nt][2 * seg + 1]);
                         }
                     }
-                }
+                    // (256 * hi-digit sum + lo-digit sum) * 2^(e_k - 129) * 2^(qe - 14) * scale, per block
+                    float s0[NT], s1[NT];
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    sc[mt][nt][0] = ((acc[nt][0][0] + acc[nt][0][1]) + (acc[nt][1][0] + acc[nt][1][1])) * kfac[nt];
-                    sc[mt][nt][1] = ((acc[nt][0][2] + acc[nt][0][3]) + (acc[nt][1][2] + acc[nt][1][3])) * kfac[nt];
+                    for (int nt = 0; nt < NT; ++nt) s0[nt] = s1[nt] = 0.f;
+#pragma unroll
+                    for (int k = 0; k < NBLK; ++k) {
+                        const float w0 = lutf[st[kei_off + mt * 16 * ROW_E + k]];
+                        const float w1 = lutf[st[kei_off + (mt * 16 + 8) * ROW_E + k]];
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const float f0 = __int2float_rn(256 * acc[nt][k][0] + acc[nt][k][1]);
+                            const float f1 = __int2float_rn(256 * acc[nt][k][2] + acc[nt][k][3]);
+                            s0[nt] = fmaf(f0, w0 * qfac[nt][k], s0[nt]);
+                            s1[nt] = fmaf(f1, w1 * qfac[nt][k], s1[nt]);
+                        }
+                    }
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) { sc[mt][nt][0] = s0[nt]; sc[mt][nt][1] = s1[nt]; }
+                } else {
+                    const uint4 xa = *reinterpret_cast<const uint4*>(st + k_off + mt * 16 * ROW_M);
+                    const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off + (mt * 16 + 8) * ROW_M);
+                    const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wb[4] = {xb.x, xb.y, xb.z, xb.w};
+                    uint2 la[NBK], lb[NBK];
+    #pragma unroll
+                    for (int k = 0; k < NBK; ++k) {
+                        la[k] = lutk[st[ke_off + mt * 16 * ROW_E + k]];
+                        lb[k] = lutk[st[ke_off + (mt * 16 + 8) * ROW_E + k]];
+                    }
+                    float acc[NT][2][4];
+    #pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int kb = (NBK == 2) ? (i >> 1) : 0;
+                        // bytes 4i..4i+3 of the lane chunk: kind 1 by byte permute, kind 2 by one logic op
+                        const uint32_t a1_01 = prmt(wa[i], kMagic, 0x4140u), a1_23 = prmt(wa[i], kMagic, 0x4342u);
+                        const uint32_t b1_01 = prmt(wb[i], kMagic, 0x4140u), b1_23 = prmt(wb[i], kMagic, 0x4342u);
+                        const uint32_t a2_01 = lop3<0x6A>(a1_01, 0xFF0FFF0Fu, 0x00800080u), a2_23 = lop3<0x6A>(a1_23, 0xFF0FFF0Fu, 0x00800080u);
+                        const uint32_t b2_01 = lop3<0x6A>(b1_01, 0xFF0FFF0Fu, 0x00800080u), b2_23 = lop3<0x6A>(b1_23, 0xFF0FFF0Fu, 0x00800080u);
+                        const uint32_t A0 = fma_f16x2(a1_01, la[kb].x, la[kb].y), A1 = fma_f16x2(b1_01, lb[kb].x, lb[kb].y);
+                        const uint32_t A2 = fma_f16x2(a2_01, la[kb].x, la[kb].y), A3 = fma_f16x2(b2_01, lb[kb].x, lb[kb].y);
+                        const uint32_t B0 = fma_f16x2(a1_23, la[kb].x, la[kb].y), B1 = fma_f16x2(b1_23, lb[kb].x, lb[kb].y);
+                        const uint32_t B2 = fma_f16x2(a2_23, la[kb].x, la[kb].y), B3 = fma_f16x2(b2_23, lb[kb].x, lb[kb].y);
+    #pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const uint2 q0 = qf[nt][2 * i], q1 = qf[nt][2 * i + 1];
+                            if (i == 0) {
+                                mma_f16_first(acc[nt][0], A0, A1, A2, A3, q0.x, q0.y);
+                                mma_f16_first(acc[nt][1], B0, B1, B2, B3, q1.x, q1.y);
+                            } else {
+                                mma_f16(acc[nt][0], A0, A1, A2, A3, q0.x, q0.y);
+                                mma_f16(acc[nt][1], B0, B1, B2, B3, q1.x, q1.y);
+                            }
+                        }
+                    }
+    #pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        sc[mt][nt][0] = ((acc[nt][0][0] + acc[nt][0][1]) + (acc[nt][1][0] + acc[nt][1][1])) * kfac[nt];
+                        sc[mt][nt][1] = ((acc[nt][0][2] + acc[nt][0][3]) + (acc[nt][1][2] + acc[nt][1][3])) * kfac[nt];
+                    }
                 }
                 if (!FULL) {       // select, not arithmetic: rows past the end may hold anything
 #pragma unroll
@@ -577,11 +748,12 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
         if (per_sm < 1 || n_sm < 1) return KVBFP_ERR_CUDA;
         resident[dev] = per_sm * n_sm;
     }
-    // per-query exponents sit behind the fragments in the query region of the workspace
-    int32_t* qexp = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
+    // per-query exponents and biases (8 words each) sit behind the fragments in the query region of the workspace
+    int32_t* qmeta = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
                                                (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
-    make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qexp);
+    if (N >= 32) make_qfrag4i<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
+    else make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
     KVBFP_LAUNCH_CHECK("make_qfrag4");
     const int64_t n_items = (int64_t)a.fmt.batch * a.fmt.n_kv_heads * a.n_chunks;
     const int64_t want = (n_items + kWarps - 1) / kWarps;
@@ -590,7 +762,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma4<N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(a, qexp);
+    decode_mma4<N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(a, qmeta);
     KVBFP_LAUNCH_CHECK("decode_mma4");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;

@@ -109,6 +109,11 @@ __device__ __forceinline__ uint32_t pack_f16x2_rn(float lo, float hi) {
     asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
 }
+// Integer MMA: 16 x 16 unsigned bytes (A) times 16 x 8 signed bytes (B), 32-bit accumulate.
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0) {
+    asm("mma.sync.aligned.m16n8k16.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(b0));
+}
 __device__ __forceinline__ uint32_t vmaxu4(uint32_t a, uint32_t b) { return __vmaxu4(a, b); }
 
 }  // namespace kvbfp
