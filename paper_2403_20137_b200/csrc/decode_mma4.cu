@@ -426,7 +426,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
     const int v_off = G_::VM_OFF + t * ROW_M + g * 8;
     const int ve_off = G_::VE_OFF + t * ROW_E + (16 * g) / N;
     const int src_lo = 4 * t + (g >> 1), src_hi = 4 * (t + 4) + (g >> 1);
-    const bool odd_col = (g & 1) != 0;
+    const uint32_t half_sel = (g & 1) ? 0x7632u : 0x5410u;     // odd columns carry the lo halves
 
     int stage = 0;
     uint32_t parity = 0;
@@ -631,17 +631,17 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                     const float p0 = ex2_approx(sc[mt][nt][0] - m_run[nt]);
                     const float p1 = ex2_approx(sc[mt][nt][1] - m_run[nt]);
                     l_run[nt] += p0 + p1;
-                    const float v0 = __shfl_sync(0xffffffffu, p0, src_lo);   // token t
-                    const float v1 = __shfl_sync(0xffffffffu, p0, src_hi);   // token t+4
-                    const float v2 = __shfl_sync(0xffffffffu, p1, src_lo);   // token t+8
-                    const float v3 = __shfl_sync(0xffffffffu, p1, src_hi);   // token t+12
-                    // hi half = the value cut to 11 significant bits (exact in fp16); lo half = the rest
-                    const float h0 = __uint_as_float(__float_as_uint(v0) & 0xffffe000u);
-                    const float h1 = __uint_as_float(__float_as_uint(v1) & 0xffffe000u);
-                    const float h2 = __uint_as_float(__float_as_uint(v2) & 0xffffe000u);
-                    const float h3 = __uint_as_float(__float_as_uint(v3) & 0xffffe000u);
-                    pb[nt][0] = odd_col ? pack_f16x2_rn(v0 - h0, v1 - h1) : pack_f16x2_rn(h0, h1);
-                    pb[nt][1] = odd_col ? pack_f16x2_rn(v2 - h2, v3 - h3) : pack_f16x2_rn(h2, h3);
+                    // (hi, lo) fp16 halves of each weight, packed in one register before they travel: hi = the
+                    // value cut to 11 significant bits (exact in fp16), lo = the rest
+                    const float h0 = __uint_as_float(__float_as_uint(p0) & 0xffffe000u);
+                    const float h1 = __uint_as_float(__float_as_uint(p1) & 0xffffe000u);
+                    const uint32_t w0 = pack_f16x2_rn(h0, p0 - h0), w1 = pack_f16x2_rn(h1, p1 - h1);
+                    const uint32_t v0 = __shfl_sync(0xffffffffu, w0, src_lo);   // token t
+                    const uint32_t v1 = __shfl_sync(0xffffffffu, w0, src_hi);   // token t+4
+                    const uint32_t v2 = __shfl_sync(0xffffffffu, w1, src_lo);   // token t+8
+                    const uint32_t v3 = __shfl_sync(0xffffffffu, w1, src_hi);   // token t+12
+                    pb[nt][0] = prmt(v0, v1, half_sel);      // this column's half of tokens (t, t+4)
+                    pb[nt][1] = prmt(v2, v3, half_sel);      // and of tokens (t+8, t+12)
                 }
                 // V pieces: bytes [8g, 8g+8) (slots 16g..16g+15) of tokens t, t+4, t+8, t+12 of this row tile
                 uint2 vw[4];
