@@ -503,13 +503,6 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                 if (KI) {
                     // ---- integer path: bytes as they are (kind 1) and 16 x low nibble (kind 2), per 16-byte segment
                     int acc[NT][NBLK][4];
-#pragma unroll
-                    for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-                        for (int k = 0; k < NBLK; ++k) {      // the offsets' constant contribution goes in up front
-                            acc[nt][k][0] = 0; acc[nt][k][1] = -qbias[nt][k];
-                            acc[nt][k][2] = 0; acc[nt][k][3] = -qbias[nt][k];
-                        }
                     const uint8_t* pa = st + k_off + mt * 16 * ROW_M;
 #pragma unroll
                     for (int seg = 0; seg < 4; ++seg) {
@@ -519,7 +512,10 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                         constexpr int SEG_PER_BLK = 4 / NBLK;
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
-                            mma_u8s8(acc[nt][seg / SEG_PER_BLK], wa, wb, qi8[nt][2 * seg]);
+                            if (seg % SEG_PER_BLK == 0)   // first MMA of a block: the offsets' constant contribution goes in as C
+                                mma_u8s8_first(acc[nt][seg / SEG_PER_BLK], wa, wb, qi8[nt][2 * seg], 0, -qbias[nt][seg / SEG_PER_BLK]);
+                            else
+                                mma_u8s8(acc[nt][seg / SEG_PER_BLK], wa, wb, qi8[nt][2 * seg]);
                             mma_u8s8(acc[nt][seg / SEG_PER_BLK], la, lb, qi8[nt][2 * seg + 1]);
                         }
                     }
