@@ -30,22 +30,45 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
     float m = -INFINITY, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = 0; i < nc;) {
-        const float* p = base + (int64_t)i * kPartStride;
-        const float mi = p[D], li = p[D + 1];
-        const float4 o = *reinterpret_cast<const float4*>(p + lane * 4);
-        const float mn = fmaxf(m, mi);
-        const float a1 = (m == -INFINITY) ? 0.f : exp2f(m - mn), a2 = (mi == -INFINITY) ? 0.f : exp2f(mi - mn);
-        acc.x = acc.x * a1 + a2 * o.x; acc.y = acc.y * a1 + a2 * o.y;
-        acc.z = acc.z * a1 + a2 * o.z; acc.w = acc.w * a1 + a2 * o.w;
-        l = l * a1 + a2 * li;
-        m = mn;
-        if (n_warps == 0) {
-            ++i;
-        } else {                                     // next partial of the pair: where the next range starts
-            const long long item = first + i;
-            const long long w = ((item + 1) * n_warps - 1) / n_items;      // range that holds this item
-            i = (int)(((w + 1) * n_items) / n_warps - first);
+        // up to eight partials at a time: first their slots (integer arithmetic only), then all loads together
+        int slot[8];
+        int cnt = 0;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            slot[k] = i;
+            if (i < nc) {
+                ++cnt;
+                if (n_warps == 0) {
+                    ++i;
+                } else {                             // next partial of the pair: where the next range starts
+                    const long long item = first + i;
+                    const long long w = ((item + 1) * n_warps - 1) / n_items;      // range that holds this item
+                    i = (int)(((w + 1) * n_items) / n_warps - first);
+                }
+            }
         }
+        float mi[8], li[8];
+        float4 oi[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float* p = base + (int64_t)(k < cnt ? slot[k] : 0) * kPartStride;
+            mi[k] = (k < cnt) ? p[D] : -INFINITY;
+            li[k] = (k < cnt) ? p[D + 1] : 0.f;
+            oi[k] = (k < cnt) ? *reinterpret_cast<const float4*>(p + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float mn = m;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) mn = fmaxf(mn, mi[k]);
+        const float a1 = (m == -INFINITY) ? 0.f : exp2f(m - mn);
+        acc.x *= a1; acc.y *= a1; acc.z *= a1; acc.w *= a1;
+        l *= a1;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const float a2 = (mi[k] == -INFINITY) ? 0.f : exp2f(mi[k] - mn);
+            acc.x += a2 * oi[k].x; acc.y += a2 * oi[k].y; acc.z += a2 * oi[k].z; acc.w += a2 * oi[k].w;
+            l += a2 * li[k];
+        }
+        m = mn;
     }
     const float inv = (l > 0.f) ? 1.f / l : 0.f;
     float* dst = out + (int64_t)row * D;

@@ -180,86 +180,83 @@ __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t*
     }
 }
 
-// Integer variant (blocks of 32 slots or more).  One warp per (batch, kv head, n-tile).  The coefficients of
+// Integer variant (blocks of 32 slots or more).  One 128-thread block per (batch, kv head, n-tile).  The coefficients of
 // every block are cast to C = round(c * 2^(14 - qe)) with the block's own exponent qe and written as two signed
 // byte digits, C = 256 * d1 + d0, in the B-fragment order of the byte MMA: fragment m = 2 * seg + kind covers the
 // bytes [16 seg, 16 seg + 16) of a row; lane (g, t) holds bytes 4t..4t+3 for column g = (query g/2, digit g%2:
 // 0 = d1, 1 = d0).  qmeta[query][2 blk] = qe, qmeta[query][2 blk + 1] = 136 * sum(C of kind 1) + 128 * sum(C of kind 2).
-__global__ void __launch_bounds__(32) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
-    const int N = a.fmt.block;
-    const int lane = threadIdx.x, gp = lane >> 2, tp = lane & 3;
+__global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
+    // one thread per slot, the four query heads of the n-tile in turn
+    const int N = a.fmt.block, nblk = D / N;
+    const int s = threadIdx.x, blk = s / N;
     const int item = blockIdx.x;
     const int nt = item % NT, hk = (item / NT) % a.fmt.n_kv_heads, b = item / NT / a.fmt.n_kv_heads;
     const int G = a.n_q_heads / a.fmt.n_kv_heads;
-    __shared__ float sq[4][D];       // pi(q) of the four query heads of this n-tile, then the coefficients
-    __shared__ int sC[4][D];         // fixed-point coefficients
-    for (int i = lane; i < 4 * D; i += 32) {
-        const int qq = 4 * nt + i / D, slot = i % D;
-        float v = 0.f;
-        if (qq < G) {
-            const int ch = a.perm_k ? (a.perm_k[hk * D + slot] & (D - 1)) : slot;
-            const int64_t idx = ((int64_t)b * a.n_q_heads + hk * G + qq) * D + ch;
-            v = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
+    __shared__ int sC[4][D];              // fixed-point coefficients
+    __shared__ uint32_t smax[2][4][8];    // block maxima: [0] of q (BFP query cast), [1] of the coefficients
+    __shared__ int sbias[4][8];
+    if (s < 64) reinterpret_cast<uint32_t*>(smax)[s] = 0u;
+    if (s < 32) reinterpret_cast<int*>(sbias)[s] = 0;
+    __syncthreads();
+    const int ch = a.perm_k ? (a.perm_k[hk * D + s] & (D - 1)) : s;
+    float v[4];
+#pragma unroll
+    for (int qq = 0; qq < 4; ++qq) {
+        v[qq] = 0.f;
+        if (4 * nt + qq < G) {
+            const int64_t idx = ((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * D + ch;
+            v[qq] = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
         }
-        sq[i / D][slot] = v;
     }
-    __syncwarp();
-    const int nblk = D / N;
     if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
-        for (int i = lane; i < 4 * nblk; i += 32) {
-            float* blk = &sq[i / nblk][(i % nblk) * N];
-            uint32_t am = 0;
-            for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(blk[j]) & 0x7fffffffu);
-            int e8 = (int)(am >> 23);
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq) atomicMax(&smax[0][qq][blk], __float_as_uint(v[qq]) & 0x7fffffffu);
+        __syncthreads();
+#pragma unroll
+        for (int qq = 0; qq < 4; ++qq) {
+            int e8 = (int)(smax[0][qq][blk] >> 23);
             if (e8 == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e8 = 254; }
             const int k = 127 - e8 + 6, k1 = k >> 1, k2 = k - k1;
-            const float w = unit_weight(e8, 8);
-            for (int j = 0; j < N; ++j) {
-                float tv = (blk[j] * pow2i(k1)) * pow2i(k2);
-                blk[j] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * w;
-            }
+            const float tv = (v[qq] * pow2i(k1)) * pow2i(k2);
+            v[qq] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * unit_weight(e8, 8);
         }
-        __syncwarp();
     }
-    // coefficients in place: slot 2j+1 <- c1 = q_hi/16 (kind 1: whole byte), slot 2j <- c2 = (q_lo - q_hi/16)/16
+    // coefficients: odd slot 2j+1 <- c1 = q_hi/16 (kind 1: whole byte), even slot 2j <- c2 = (q_lo - q_hi/16)/16
     // (kind 2: 16 x low nibble).  Both multiply operands that carry a factor 16, so they have the same size and
     // one block exponent serves both without losing bits of either.
-    for (int i = lane; i < 4 * (D / 2); i += 32) {
-        float* pr2 = &sq[i / (D / 2)][2 * (i % (D / 2))];
-        const float c1 = pr2[1] * 0.0625f, c2 = (pr2[0] - c1) * 0.0625f;
-        pr2[0] = c2;
-        pr2[1] = c1;
+    float c[4];
+#pragma unroll
+    for (int qq = 0; qq < 4; ++qq) {
+        const float other = __shfl_xor_sync(0xffffffffu, v[qq], 1);
+        c[qq] = (s & 1) ? v[qq] * 0.0625f : (v[qq] - other * 0.0625f) * 0.0625f;
+        atomicMax(&smax[1][qq][blk], __float_as_uint(c[qq]) & 0x7fffffffu);
     }
-    __syncwarp();
-    // per (query, block): exponent, fixed-point cast, bias
-    for (int i = lane; i < 4 * nblk; i += 32) {
-        const int qq = i / nblk, blk = i % nblk;
-        const float* c = &sq[qq][blk * N];
-        uint32_t am = 0;
-        for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(c[j]) & 0x7fffffffu);
+    __syncthreads();
+#pragma unroll
+    for (int qq = 0; qq < 4; ++qq) {
+        const uint32_t am = smax[1][qq][blk];
         int e = (int)(am >> 23);
         if (e == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e = 254; }
         const int qe = (am == 0) ? 0 : e - 126;               // |c| * 2^-qe < 1
         const int sh = 14 - qe, h1 = sh / 2, h2 = sh - h1;    // two exact factors (sh in [-114, 140])
-        const float f1 = pow2i(h1), f2 = pow2i(h2);
-        int bias = 0;
-        for (int j = 0; j < N; ++j) {
-            const int C = __float2int_rn((c[j] * f1) * f2);
-            sC[qq][blk * N + j] = C;
-            bias += ((j & 1) ? 136 : 128) * C;
-        }
-        if (4 * nt + qq < G) {
-            int32_t* m = qmeta + ((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8;
-            m[2 * blk] = qe;
-            m[2 * blk + 1] = bias;
-        }
+        const int C = __float2int_rn((c[qq] * pow2i(h1)) * pow2i(h2));
+        sC[qq][s] = C;
+        atomicAdd(&sbias[qq][blk], ((s & 1) ? 136 : 128) * C);
+        if (s % N == 0 && 4 * nt + qq < G)
+            qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * blk] = qe;
     }
-    __syncwarp();
+    __syncthreads();
+    if (s < 4 * nblk) {
+        const int qq = s / nblk, k = s % nblk;
+        if (4 * nt + qq < G) qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * k + 1] = sbias[qq][k];
+    }
+    // fragments: word (m, lane) for m = 0..7; thread s writes (m = s / 32, lane = s % 32) and (m + 4, lane)
+    const int lane = s & 31, gp = lane >> 2, tp = lane & 3;
     const int qq = gp >> 1, digit = gp & 1, qi = 4 * nt + qq;
     uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
 #pragma unroll
-    for (int m = 0; m < 8; ++m) {
-        const int seg = m >> 1, kind = m & 1;
+    for (int mm = 0; mm < 2; ++mm) {
+        const int m = (s >> 5) + 4 * mm, seg = m >> 1, kind = m & 1;
         uint32_t reg = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
@@ -748,7 +745,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
     int32_t* qmeta = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
                                                (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
-    if (N >= 32) make_qfrag4i<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
+    if (N >= 32) make_qfrag4i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
     else make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
     KVBFP_LAUNCH_CHECK("make_qfrag4");
     const int64_t n_items = (int64_t)a.fmt.batch * a.fmt.n_kv_heads * a.n_chunks;
