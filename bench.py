@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": None, "sources_sha256": None}}
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 141.2573, "sources_sha256": "48bf2a1330fed08ce19a8d1dded840160d5ad39cc313147133db387fc06b856c"}}
 KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
 
 
