@@ -210,6 +210,39 @@ def run_reference(args, w, rank):
     }))
 
 
+def sweep_config5(B, dev):
+    """Prefill/append and calibration sweep: 8 KV heads x 128, 65536 new bf16 tokens with the outlier law,
+    calibration (max-abs + argsort) over 2^20 tokens, append throughput and key MSE with/without K-sort for
+    blocks 16/32/64 x mantissas 4/6/8."""
+    w = W.CONFIGS[5]
+    H, d, T = w.n_kv_heads, w.head_dim, w.seq
+    out = {}
+    calib = W.make_calibration(w, device=dev)                       # [2^20, 8, 128] bf16 = 2 GiB
+    _, perm, _ = B.calibrate(calib, H, d)
+    ms = timed(lambda: B.calibrate(calib, H, d), reps=3)
+    out["calibrate"] = {"tokens": int(calib.shape[0]), "ms": ms, "GB/s": calib.numel() * 2 / ms / 1e6}
+    del calib
+    k, v = W.make_kv(w, n_tokens=T, device=dev, batch=1)             # [1, 65536, 8, 128]
+    z = torch.zeros(1, dtype=torch.int32, device=dev)
+    ref = k[0, :4096, 0].float()
+    rows = 2 * T * H
+    fm = {}
+    for n in (16, 32, 64):
+        for p in (4, 6, 8):
+            c = B.Cache(1, H, d, T, n, p, device=dev)
+            B.append(c, k, v, z, perm_k=perm)
+            ms = timed(lambda: B.append(c, k, v, z, perm_k=perm), reps=3)
+            row_bytes = d * 2 + d * p // 8 + d // n
+            mse_s = float(((B.dequant(c, "k", 0, 0, 0, 4096, perm=perm) - ref) ** 2).mean())
+            B.append(c, k, None, z)
+            mse_u = float(((B.dequant(c, "k", 0, 0, 0, 4096) - ref) ** 2).mean())
+            fm[f"n{n}_p{p}"] = {"ms": ms, "GB/s": rows * row_bytes / ms / 1e6, "elements/s": rows * d / (ms * 1e-3),
+                                "key_mse_unsorted": mse_u, "key_mse_ksort": mse_s}
+            del c
+    out["append"] = fm
+    return out
+
+
 def timed(fn, reps=1):
     """Milliseconds per call of fn(), CUDA events on the current stream."""
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -240,6 +273,7 @@ def main():
     ap.add_argument("--chunk", type=int, default=0, help="tokens per sequence chunk (0 = library default)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the set-up timings and the quality report")
+    ap.add_argument("--sweep5", action="store_true", help="add the prefill/append and calibration sweep (8 KV heads, 65536 new\n                    tokens, blocks 16/32/64 x mantissas 4/6/8, calibration over 2^20 tokens) to the extras")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
     over = {k: v for k, v in (("batch", args.batch), ("seq", args.seq), ("mant_bits", args.mant_bits),
@@ -310,6 +344,8 @@ def main():
         del plain, sortd, kk, dq_p, dq_s
     k_new, v_new = k[:, S - 1:].contiguous(), v[:, S - 1:].contiguous()
     del k, v, k_pre, v_pre
+    if args.sweep5 and rank == 0:
+        extras["config5"] = sweep_config5(B, dev)
     q = W.make_q(w, device=dev)
     start_pos = torch.full((Bn,), S - 1, dtype=torch.int32, device=dev)
     seq_lens = torch.full((Bn,), S, dtype=torch.int32, device=dev)
