@@ -161,6 +161,30 @@ kvbfp_status kvbfp_dequant(const kvbfp_format* fmt, const uint8_t* mant, const u
                            int32_t b, int32_t h, int32_t t0, int32_t n_tok, const int32_t* perm,
                            void* out, kvbfp_dtype out_dt, void* stream);
 
+/*
+ * Algorithm 1 step 5 (Sec. III): rotary-embedding tables in stored (slot) order, so that rows that are already
+ * permuted can be rotated (Sec. II-D, Eq. (4)) without undoing K-sort.  Slot j of head h holds channel
+ * c = perm[h*d+j]; the tables give that channel's frequency, the slot of its rotation partner and the sine sign.
+ *   perm, inv_perm  [n_heads*head_dim] i32, both NULL for the identity
+ *   base            frequency base (10000 in RoFormer); theta_i = base^(-2i/d)
+ *   half_split      0: pairs of neighbouring channels (2i, 2i+1), the layout of Eq. (4);
+ *                   1: pairs (i, i + d/2), the layout of the open-source Llama code (footnote to Sec. III)
+ *   theta_out       [n_heads*head_dim] f64;  partner_out [n_heads*head_dim] i32;  sign_out [n_heads*head_dim] f32
+ */
+kvbfp_status kvbfp_rope_tables(const int32_t* perm, const int32_t* inv_perm, int32_t n_heads,
+                               int32_t head_dim, double base, int32_t half_split, double* theta_out,
+                               int32_t* partner_out, float* sign_out, void* stream);
+
+/*
+ * Eq. (4) in table form on rows in slot order: y[j] = x[j] cos(m theta_j) + sign_j x[partner_j] sin(m theta_j),
+ * m = positions[row].  The angle is formed in fp64; y is rounded once to `dt`.
+ *   x, y       [n_rows, n_heads, head_dim] of `dt`, y != x
+ *   positions  [n_rows] i32
+ */
+kvbfp_status kvbfp_rope_apply(const void* x, kvbfp_dtype dt, int64_t n_rows, int32_t n_heads,
+                              int32_t head_dim, const int32_t* positions, const double* theta,
+                              const int32_t* partner, const float* sign, void* y, void* stream);
+
 /* Bytes of workspace kvbfp_decode_attn needs for this cache geometry (0 on invalid arguments). */
 size_t kvbfp_decode_workspace_bytes(const kvbfp_format* fmt, int32_t n_q_heads);
 

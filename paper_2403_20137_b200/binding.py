@@ -23,7 +23,8 @@ EXPORTS = ["kvbfp_version", "kvbfp_status_string", "kvbfp_last_cuda_error", "kvb
            "kvbfp_calibrate", "kvbfp_fold_perm", "kvbfp_append", "kvbfp_dequant",
            "kvbfp_decode_workspace_bytes", "kvbfp_decode_attn", "kvbfp_device_status",
            "kvbfp_launch_count", "kvbfp_step_staging_bytes", "kvbfp_decode_step_host",
-           "kvbfp_profile_decode_events", "kvbfp_static_scratch_bytes", "kvbfp_decode_attn_static"]
+           "kvbfp_profile_decode_events", "kvbfp_static_scratch_bytes", "kvbfp_decode_attn_static",
+           "kvbfp_rope_tables", "kvbfp_rope_apply"]
 
 
 class KvbfpError(RuntimeError):
@@ -96,6 +97,10 @@ def lib():
         L.kvbfp_decode_attn_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int32,
                                                C.c_void_p, C.c_void_p, C.c_float, C.c_int32, C.c_void_p,
                                                C.c_uint32, C.c_void_p]
+        L.kvbfp_rope_tables.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_double, C.c_int32,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.kvbfp_rope_apply.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -293,3 +298,25 @@ def decode_attn_static(cache, q, seq_lens, perm_k=None, inv_perm_v=None, softmax
                                           float(softmax_scale), q_mant_bits, _ptr(_dev(out, torch.float32)), flags,
                                           _stream(stream)))
     return out
+
+
+def rope_tables(perm, inv_perm, n_heads, head_dim, base=10000.0, half_split=False, device="cuda", stream=None):
+    """kvbfp_rope_tables -> (theta f64 [H, d], partner i32 [H, d], sign f32 [H, d]) in slot order."""
+    theta = torch.empty(n_heads, head_dim, dtype=torch.float64, device=device)
+    partner = torch.empty(n_heads, head_dim, dtype=torch.int32, device=device)
+    sign = torch.empty(n_heads, head_dim, dtype=torch.float32, device=device)
+    _check(lib().kvbfp_rope_tables(_ptr(_dev(perm, torch.int32)), _ptr(_dev(inv_perm, torch.int32)), n_heads, head_dim,
+                                   float(base), int(half_split), _ptr(theta), _ptr(partner), _ptr(sign), _stream(stream)))
+    return theta, partner, sign
+
+
+def rope_apply(x, positions, theta, partner, sign, stream=None):
+    """kvbfp_rope_apply: x [rows, H, d] in slot order, positions i32 [rows] -> rotated rows of the same dtype."""
+    x = _dev(x)
+    y = torch.empty_like(x)
+    n_heads, head_dim = x.shape[-2], x.shape[-1]
+    n_rows = x.numel() // (n_heads * head_dim)
+    _check(lib().kvbfp_rope_apply(_ptr(x), _dt(x), n_rows, n_heads, head_dim, _ptr(_dev(positions, torch.int32)),
+                                  _ptr(_dev(theta, torch.float64)), _ptr(_dev(partner, torch.int32)),
+                                  _ptr(_dev(sign, torch.float32)), _ptr(y), _stream(stream)))
+    return y

@@ -339,6 +339,39 @@ def test_ksort_improves_gpu_cache_quality(oracle):
     assert mse_s < 0.85 * mse_p
 
 
+# ------------------------------------------------------------------------------- permuted RoPE
+@pytest.mark.parametrize("half_split", [False, True])
+def test_rope_tables_and_apply(oracle, half_split):
+    """Algorithm 1 step 5 and Eq. (4) on the GPU against the oracle, including the identity
+    rotate-then-permute = permute-then-rotate-with-permuted-tables."""
+    rng = np.random.default_rng(12)
+    H, d, rows = 3, 128, 7
+    perm = np.stack([rng.permutation(d) for _ in range(H)]).astype(np.int32)
+    inv = np.argsort(perm, axis=1).astype(np.int32)
+    th, pa, sg = B.rope_tables(dev(torch.from_numpy(perm)), dev(torch.from_numpy(inv)), H, d, 10000.0, half_split)
+    x = rng.standard_normal((rows, H, d)).astype(np.float32)                 # original channel order
+    pos = np.array([0, 1, 2, 77, 4095, 32767, 100000], dtype=np.int32)
+    xs = np.stack([x[:, h, perm[h]] for h in range(H)], axis=1)             # slot order
+    y = host(B.rope_apply(dev(torch.from_numpy(xs)), dev(torch.from_numpy(pos)), th, pa, sg)).astype(np.float64)
+    t0, p0, s0 = oracle.rope_tables(d, 10000.0, half_split)
+    for h in range(H):
+        tp, pp, sp = oracle.rope_permute_tables(perm[h], inv[h], t0, p0, s0)
+        assert np.allclose(host(th[h]), tp, rtol=1e-14, atol=0)
+        assert np.array_equal(host(pa[h]), pp) and np.array_equal(host(sg[h]).astype(np.float64), sp)
+        for r in range(rows):
+            ref_slot = oracle.rope_apply(xs[r, h].astype(np.float64), float(pos[r]), tp, pp, sp)
+            assert np.allclose(y[r, h], ref_slot, rtol=0, atol=2e-6)
+            ref_orig = oracle.rope_apply(x[r, h].astype(np.float64), float(pos[r]), t0, p0, s0)
+            assert np.allclose(y[r, h], ref_orig[perm[h]], rtol=0, atol=2e-6)          # commutes with the permutation
+    # identity tables and bf16 rows
+    th1, pa1, sg1 = B.rope_tables(None, None, H, d, 10000.0, half_split)
+    xb = torch.from_numpy(x).to(torch.bfloat16)
+    yb = host(B.rope_apply(dev(xb), dev(torch.from_numpy(pos)), th1, pa1, sg1).float()).astype(np.float64)
+    for r in (3, 5):
+        ref = oracle.rope_apply(xb[r, 1].float().numpy().astype(np.float64), float(pos[r]), t0, p0, s0)
+        assert np.allclose(yb[r, 1], ref, rtol=2 ** -8, atol=1e-3)
+
+
 # ------------------------------------------------------------------------------- full-size workloads
 def _full_size_case(oracle, cfg, sample_pairs):
     """The benchmark's own launch (full batch, full sequence, library-chosen chunking) with inputs drawn on
