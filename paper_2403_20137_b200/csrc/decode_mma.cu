@@ -16,9 +16,10 @@
 // Output: O^T[16 slots x 8 cols] += V^T[16 slots x 16 tokens] . P^T[16 tokens x 8 cols], with the
 // softmax weights split into hi/lo halves the same way.  Accumulators are fp32.
 //
-// The integer pipe (logic ops, shifts, byte permutes) is what limits this kernel, so half of the
-// shifts are issued as multiply-high on the multiply-add pipe and block weights come from a
-// 256-entry table in shared memory instead of being rebuilt from the exponent byte.
+// The integer pipe (logic ops, shifts, byte permutes) is what limits this kernel: every field is
+// extracted with one three-input logic instruction and block weights come from a 256-entry table in
+// shared memory instead of being rebuilt from the exponent byte.  (Issuing shifts as multiply-high on
+// the multiply-add pipe was measured slower on B200; the switch is kept, off.)
 #include <math.h>
 
 #include "decode.cuh"

@@ -1,4 +1,5 @@
-// Decode attention over a 4-bit BFP cache with fp16 tensor-core MMAs, two mantissas per operand element
+// Decode attention over a 4-bit BFP cache: integer tensor-core MMAs for the scores, fp16 tensor-core MMAs
+// with two mantissas per operand element for P.V
 // (Sec. III par. 2 of the paper: keys are read back from the cache and multiplied with pi(q);
 // Sec. II-B: a block's values are integer mantissas times one power of two).
 //
@@ -12,8 +13,8 @@
 // There is no block-wide barrier in the loop and no cluster multicast.
 //
 // Unpacking is what limits this kernel (integer-pipe instructions, not memory).  A packed byte holds
-// two mantissas in excess-8 code: B = 16*(M_hi+8) + (M_lo+8).  fp16 has a 10-bit
-// fraction, so the whole byte can be put under the bits of 1024.0 with one byte permute: the element
+// two mantissas in excess-8 code: B = 16*(M_hi+8) + (M_lo+8).  fp16 path (P.V always; scores only for
+// blocks of 16): fp16 has a 10-bit fraction, so the whole byte can be put under the bits of 1024.0 with one byte permute: the element
 // 1024 + B.  A second element with the high nibble masked away and bit 7 set, 1024 + 128 + (M_lo+8),
 // comes from one logic op.  One f16x2 fma per register with the block's power of two removes the
 // common bias 1160 and applies the weight, exactly:
@@ -27,17 +28,18 @@
 // Scores for blocks of 32 slots or more use the integer tensor-core path instead (Sec. II-B of the paper:
 // the inner product of two BFP blocks is an integer product plus an exponent addition).  The packed
 // bytes are fed to an unsigned-byte x signed-byte MMA as they are (kind 1) and with the low nibble moved
-// up (kind 2 = 16 x low nibble): two integer ops per packed word and no conversion at all.  The query coefficients of
+// up (kind 2 = 16 x low nibble): two integer ops per packed word and no conversion at all.  The query
+// coefficients c1 = q_hi/16 and c2 = (q_lo - q_hi/16)/16 (both multiply operands that carry a factor 16) of
 // each block are cast to 15-bit fixed point with the block's own exponent and split into two signed
 // byte digits, which sit in two MMA columns; the two 32-bit sums of a (token, block) are recombined
 // exactly, the constant contribution of the offsets (136 per kind-1 byte, 128 per kind-2 byte) was put
 // into the accumulator beforehand, and one fp32 multiply-add applies 2^(e_k + e_q) per (token, block).
 //
-// Range.  fp16 cannot hold 2^e for every exponent byte, so each run first takes the largest K and V
-// exponent byte of its rows (D_k, D_v) and uses the weights 2^(e - D + 5): the largest block gets
+// Range of the fp16 path.  fp16 cannot hold 2^e for every exponent byte, so each run first takes the largest
+// exponent byte D of its rows (of V, and of K when the scores use fp16) and uses the weights 2^(e - D + 5): the largest block gets
 // 2^5 (the bias product 1160 * 2^5 still fits fp16), blocks more than 2^29 below the largest one of
 // the run are flushed to zero (their contribution is below 2^-29 of it), and the common factor
-// 2^(D - 134) is applied in fp32 to the scores and to the partial output.  The weights come from a
+// 2^(D - 134) is applied in fp32 to the partial output (and to fp16 scores).  The weights come from a
 // shared-memory table addressed by exponent byte from a per-run base, so the subtraction costs
 // nothing.  q and the softmax weights are carried as (hi, lo) fp16 pairs (q after a per-head
 // power-of-two normalisation), accumulation is fp32.
