@@ -8,14 +8,15 @@ namespace kvbfp {
 namespace {
 
 // One warp per (batch, query head): out = sum_i 2^(m_i - m) o_i / sum_i 2^(m_i - m) l_i over the partial
-// results of the row.  n_warps == 0: every chunk that holds tokens has its own partial.  n_warps > 0:
-// the items (pair-major chunks) were cut into n_warps contiguous ranges and each range wrote one partial
-// per (batch, kv head) it touches, at the slot of the first chunk it covers there; the same integer
-// arithmetic as in the kernel finds those slots.
+// results of the row.  n_warps == 0: every chunk that holds tokens has its own partial (item = chunk).
+// n_warps > 0: the items (pair-major pieces of item_tokens tokens) were cut into n_warps contiguous ranges and
+// each range wrote one partial per (batch, kv head) it touches, at the slot of the chunk in which its first
+// item there lies; the same integer arithmetic as in the kernel finds those slots.
 __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ partials, const int32_t* __restrict__ seq_lens,
                                                  const int32_t* __restrict__ inv_perm_v, float* __restrict__ out,
                                                  int n_rows, int n_q_heads, int group, int n_chunks, int chunk,
-                                                 int len_cap, int n_warps, long long n_items) {
+                                                 int len_cap, int n_warps, int item_tokens, int items_per_pair,
+                                                 long long n_items) {
     constexpr int D = kHeadDim;
     __shared__ float so[4][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -24,9 +25,9 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
     const int b = row / n_q_heads, hq = row % n_q_heads;
     int len = seq_lens[b];
     len = len < 0 ? 0 : (len > len_cap ? len_cap : len);
-    const int nc = (len + chunk - 1) / chunk;        // chunks that hold tokens
+    const int nc = (len + item_tokens - 1) / item_tokens;        // items that hold tokens
     const float* base = partials + (int64_t)row * n_chunks * kPartStride;
-    const long long first = ((long long)b * (n_q_heads / group) + hq / group) * n_chunks;   // first item of the pair
+    const long long first = ((long long)b * (n_q_heads / group) + hq / group) * items_per_pair;   // first item of the pair
     float m = -INFINITY, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = 0; i < nc;) {
@@ -51,7 +52,7 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
         float4 oi[8];
 #pragma unroll
         for (int k = 0; k < 8; ++k) {
-            const float* p = base + (int64_t)(k < cnt ? slot[k] : 0) * kPartStride;
+            const float* p = base + (int64_t)(k < cnt ? partial_slot(slot[k], item_tokens, chunk, n_chunks) : 0) * kPartStride;
             mi[k] = (k < cnt) ? p[D] : -INFINITY;
             li[k] = (k < cnt) ? p[D + 1] : 0.f;
             oi[k] = (k < cnt) ? *reinterpret_cast<const float4*>(p + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
@@ -175,15 +176,20 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
     a.mulhi4 = 1u << 28; a.mulhi8 = 1u << 24; a.mulhi12 = 1u << 20;
 
     cudaStream_t s = (cudaStream_t)stream;
-    int n_warps = 0;
+    a.item_tokens = a.chunk;
+    a.items_per_pair = a.n_chunks;
+    Split split;
+    split.item_tokens = a.chunk;
+    split.items_per_pair = a.n_chunks;
     if (impl == KVBFP_DECODE_SIMT) st = launch_decode_simt(a, s);
-    else if (use_mma4) st = launch_decode_mma4(a, s, &n_warps);
+    else if (use_mma4) st = launch_decode_mma4(a, s, &split);
     else st = launch_decode_mma(a, s);
     if (st != KVBFP_OK) return st;
     const int n_rows = f.batch * n_q_heads;
     lse_merge<<<(n_rows + 3) / 4, 128, 0, s>>>(a.partials, seq_lens, inv_perm_v, out, n_rows, n_q_heads, group,
-                                              a.n_chunks, a.chunk, a.len_cap, n_warps,
-                                              (long long)f.batch * f.n_kv_heads * a.n_chunks);
+                                              a.n_chunks, a.chunk, a.len_cap, split.n_warps, split.item_tokens,
+                                              split.items_per_pair,
+                                              (long long)f.batch * f.n_kv_heads * split.items_per_pair);
     KVBFP_LAUNCH_CHECK("lse_merge");
     return KVBFP_OK;
 }

@@ -26,6 +26,8 @@ struct DecodeArgs {
     int chunk;                // tokens per chunk
     int n_chunks;
     int len_cap;              // min(max_len_hint, max_seq)
+    int item_tokens;          // persistent kernel: tokens per work item (divides chunk) and items per (batch, kv head)
+    int items_per_pair;
     uint32_t* status;
     // 2^(32-k): multiplying by these and keeping the high word is a right shift by k that runs on the
     // multiply-add pipe instead of the integer pipe (passed at run time so that it stays a multiply)
@@ -34,8 +36,25 @@ struct DecodeArgs {
 
 kvbfp_status launch_decode_simt(const DecodeArgs& a, cudaStream_t s);
 kvbfp_status launch_decode_mma(const DecodeArgs& a, cudaStream_t s);    // bf16, every mantissa width
-// fp16, 4-bit mantissas, persistent: *n_warps receives the number of warps the items were split over
-kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, int* n_warps);
+// How the persistent kernel cut the work, for the merge: the items (pair-major pieces of `item_tokens` tokens,
+// `items_per_pair` per (batch, kv head)) were split into `n_warps` contiguous ranges.  n_warps == 0: no ranges,
+// every chunk has its own partial.
+struct Split {
+    int n_warps = 0;
+    int item_tokens = 0;
+    int items_per_pair = 0;
+};
+// Slot (chunk-sized, n_chunks per pair) that receives the partial of a run whose first item within its pair
+// is `item`.  Items are whole chunks, or half chunks: then two runs can start in the first chunk of a pair (one
+// that holds only item 0, the next from item 1 on), so odd items round up; ranges hold four items or more, so
+// no other two runs start within two items of each other and the clamp at the last slot is safe as well.
+__host__ __device__ __forceinline__ int partial_slot(int item, int item_tokens, int chunk, int n_chunks) {
+    if (item_tokens == chunk) return item;
+    const int s = (item + 1) >> 1;
+    return s < n_chunks ? s : n_chunks - 1;
+}
+// 4-bit mantissas: integer scores + fp16 P.V, persistent
+kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, Split* split);
 size_t qfrag_bytes(const kvbfp_format& f, int n_q_heads);
 // Events the caller asked to have recorded around the main decode kernel (nullptr = none).
 void profile_events(cudaEvent_t* start, cudaEvent_t* stop);

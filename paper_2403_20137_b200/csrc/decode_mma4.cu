@@ -318,8 +318,8 @@ __device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int la
 // The chunks of one (batch, kv head) that fall into a warp's item range.
 struct Run {
     int b, hk;
-    int chunk0;        // first chunk: its slot receives the partial result
-    int n_items;       // chunks covered (>= 1)
+    int chunk0;        // first item within the pair: the slot of the chunk it lies in receives the partial result
+    int n_items;       // items covered (>= 1)
     int n_tok;         // tokens that exist in them (0: nothing to do)
     int n_tiles;
     int64_t row0;      // first row in the planes
@@ -349,19 +349,19 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
-    const int64_t n_items = (int64_t)a.fmt.batch * Hkv * a.n_chunks;
+    const int64_t n_items = (int64_t)a.fmt.batch * Hkv * a.items_per_pair;
     const int64_t wglob = (int64_t)blockIdx.x * kWarps + warp, wtot = (int64_t)gridDim.x * kWarps;
     const int64_t i0 = wglob * n_items / wtot, i1 = (wglob + 1) * n_items / wtot;     // this warp's items
     if (i0 >= i1) return;
 
     auto get_run = [&](int64_t it) -> Run {
         Run r;
-        const int64_t pair = it / a.n_chunks;
-        r.chunk0 = (int)(it - pair * a.n_chunks);
+        const int64_t pair = it / a.items_per_pair;
+        r.chunk0 = (int)(it - pair * a.items_per_pair);
         r.hk = (int)(pair % Hkv);
         r.b = (int)(pair / Hkv);
         const int64_t left = i1 - it;
-        r.n_items = (int)(left < (int64_t)(a.n_chunks - r.chunk0) ? left : (int64_t)(a.n_chunks - r.chunk0));
+        r.n_items = (int)(left < (int64_t)(a.items_per_pair - r.chunk0) ? left : (int64_t)(a.items_per_pair - r.chunk0));
         int len = a.seq_lens[r.b];
         if (len > a.fmt.max_seq || len < 0) {
             if (lane == 0 && r.chunk0 == 0 && r.hk == 0) raise_flag(a.status, KVBFP_FLAG_POSITION);
@@ -371,8 +371,8 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
             if (lane == 0 && r.chunk0 == 0 && r.hk == 0) raise_flag(a.status, KVBFP_FLAG_LEN_HINT);
             len = a.len_cap;
         }
-        const int tok0 = r.chunk0 * a.chunk;
-        const int64_t tok1 = (int64_t)(r.chunk0 + r.n_items) * a.chunk;
+        const int tok0 = r.chunk0 * a.item_tokens;
+        const int64_t tok1 = (int64_t)(r.chunk0 + r.n_items) * a.item_tokens;
         r.n_tok = max(0, (int)min((int64_t)len, tok1) - tok0);
         r.n_tiles = (r.n_tok + kTile - 1) / kTile;
         r.row0 = pair * a.fmt.max_seq + tok0;
@@ -701,7 +701,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
             l += __shfl_xor_sync(0xffffffffu, l, 16);
             const int qi = 4 * nt + t;
             if (qi < Gq) {
-                float* dst = a.partials + (((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + qi) * a.n_chunks + cr.chunk0) * kPartStride;
+                float* dst = a.partials + (((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + qi) * a.n_chunks + partial_slot(cr.chunk0, a.item_tokens, a.chunk, a.n_chunks)) * kPartStride;
 #pragma unroll
                 for (int r4 = 0; r4 < 4; ++r4) {
                     const float w0 = o[nt][2 * r4][0] + o[nt][2 * r4][1], l0 = o[nt][2 * r4][2] + o[nt][2 * r4][3];
@@ -729,7 +729,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
 }
 
 template <int N, int NT>
-kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
+kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     using G_ = Geo4<N>;
     static int resident[64] = {0};          // thread blocks that fit the whole device, per device
     int dev = 0;
@@ -750,33 +750,44 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
     if (N >= 32) make_qfrag4i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
     else make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
     KVBFP_LAUNCH_CHECK("make_qfrag4");
-    const int64_t n_items = (int64_t)a.fmt.batch * a.fmt.n_kv_heads * a.n_chunks;
+    // Work items: one stage (kTile tokens) each when the library chose the chunking and every warp still gets
+    // at least four of them (half chunks: the ranges then differ by one stage of work at most; partial_slot()
+    // keeps the runs' partial results apart); whole chunks otherwise.
+    DecodeArgs b = a;
+    const int64_t pairs = (int64_t)a.fmt.batch * a.fmt.n_kv_heads;
+    const int fine_per_pair = (a.len_cap + kTile - 1) / kTile;
+    const bool fine = a.chunk == 2 * kTile && a.chunk == kMinChunk && pairs * fine_per_pair >= 4LL * resident[dev] * kWarps;
+    b.item_tokens = fine ? kTile : a.chunk;
+    b.items_per_pair = fine ? fine_per_pair : a.n_chunks;
+    const int64_t n_items = pairs * b.items_per_pair;
     const int64_t want = (n_items + kWarps - 1) / kWarps;
     const int grid = (int)(want < resident[dev] ? want : resident[dev]);
-    *n_warps = grid * kWarps;
+    split->n_warps = grid * kWarps;
+    split->item_tokens = b.item_tokens;
+    split->items_per_pair = b.items_per_pair;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma4<N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(a, qmeta);
+    decode_mma4<N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b, qmeta);
     KVBFP_LAUNCH_CHECK("decode_mma4");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;
 }
 
 template <int N>
-kvbfp_status launch2(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
+kvbfp_status launch2(const DecodeArgs& a, cudaStream_t s, Split* split) {
     const int G = a.n_q_heads / a.fmt.n_kv_heads;
-    return (G <= 4) ? launch3<N, 1>(a, s, n_warps) : launch3<N, 2>(a, s, n_warps);
+    return (G <= 4) ? launch3<N, 1>(a, s, split) : launch3<N, 2>(a, s, split);
 }
 
 }  // namespace
 
-kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, int* n_warps) {
+kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, Split* split) {
     switch (a.fmt.block) {
-        case 16: return launch2<16>(a, s, n_warps);
-        case 32: return launch2<32>(a, s, n_warps);
-        case 64: return launch2<64>(a, s, n_warps);
-        case 128: return launch2<128>(a, s, n_warps);
+        case 16: return launch2<16>(a, s, split);
+        case 32: return launch2<32>(a, s, split);
+        case 64: return launch2<64>(a, s, split);
+        case 128: return launch2<128>(a, s, split);
     }
     return KVBFP_ERR_UNSUPPORTED;
 }
