@@ -73,6 +73,7 @@ constexpr int kStages = KVBFP4_STAGES;
 constexpr int D = kHeadDim;
 constexpr int ROW_M = D / 2;            // 64 bytes of mantissas per token row
 constexpr int kTopShift = 5;            // weight of the run's largest block is 2^kTopShift
+constexpr int kDvHeadroom = 2;          // binades left above a tile's largest V exponent when the reference moves
 constexpr int kLutEntries = 512;        // index = exponent byte - D + 255, D = largest valid exponent byte
 
 constexpr uint32_t kMagic = 0x64646464u;        // 0x64 = high byte of fp16 1024.0
@@ -294,9 +295,9 @@ struct Geo4 {
 __device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int lane) {
     uint32_t m = 0;
     const uint4* v = reinterpret_cast<const uint4*>(p);
-    for (int i = lane; i < ((bytes + 15) >> 4); i += 32) {
-        uint4 x = __ldg(v + i);
-        const int left = bytes - 16 * i;             // valid bytes in this vector (may exceed 16)
+    const int n_vec = (bytes + 15) >> 4;
+    auto masked = [&](uint4 x, int i) -> uint32_t {
+        const int left = bytes - 16 * i;                 // valid bytes in this vector (may exceed 16)
         if (left < 16) {
             uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
@@ -306,7 +307,18 @@ __device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int la
             }
             x = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        m = vmaxu4(vmaxu4(m, x.x), vmaxu4(x.y, vmaxu4(x.z, x.w)));
+        return vmaxu4(vmaxu4(x.x, x.y), vmaxu4(x.z, x.w));
+    };
+    // eight vectors per lane in flight at a time: the pass is latency, not bandwidth
+    for (int i0 = lane; i0 < n_vec; i0 += 8 * 32) {
+        uint4 x[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = i0 + 32 * u;
+            x[u] = i < n_vec ? __ldg(v + i) : make_uint4(0u, 0u, 0u, 0u);
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) m = vmaxu4(m, masked(x[u], i0 + 32 * u));
     }
 #pragma unroll
     for (int off = 16; off; off >>= 1) m = vmaxu4(m, __shfl_xor_sync(0xffffffffu, m, off));
@@ -334,26 +346,11 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
     constexpr int NBLK = KI ? D / N : 1;              // blocks of a row (integer path)
     extern __shared__ __align__(128) uint8_t smem[];
 
-    // weight table: entry i = (2^(i - 255 + kTopShift) twice as f16x2, the same times -1160); entries
-    // above 255 belong to rows that are masked later (past the end of the run) and only have to exist
-    uint2* lut = reinterpret_cast<uint2*>(smem + G_::LUT_OFF);
-    for (int i = threadIdx.x; i < kLutEntries; i += kWarps * 32) {
-        const uint32_t s2 = (i <= 255 ? pow2_f16(i - 255 + kTopShift) : 0u) * 0x00010001u;
-        lut[i] = make_uint2(s2, mul_f16x2(s2, kBias));
-    }
-    // integer score path: 2^(e - 129), the true weight of a mantissa unit, as fp32 (no range issue there)
-    float* lutf = reinterpret_cast<float*>(smem + G_::LUTF_OFF);
-    if (KI)
-        for (int i = threadIdx.x; i < 256; i += kWarps * 32) lutf[i] = unit_weight(i, 4);
-    __syncthreads();
-
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
     const int64_t n_items = (int64_t)a.fmt.batch * Hkv * a.items_per_pair;
     const int64_t wglob = (int64_t)blockIdx.x * kWarps + warp, wtot = (int64_t)gridDim.x * kWarps;
     const int64_t i0 = wglob * n_items / wtot, i1 = (wglob + 1) * n_items / wtot;     // this warp's items
-    if (i0 >= i1) return;
-
     auto get_run = [&](int64_t it) -> Run {
         Run r;
         const int64_t pair = it / a.items_per_pair;
@@ -418,6 +415,21 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
     };
     for (int s = 0; s < kStages; ++s) issue_next(s);
 
+    // (the tables are filled while the first copies are in flight)
+    // weight table: entry i = (2^(i - 255 + kTopShift) twice as f16x2, the same times -1160); entries
+    // above 255 belong to rows that are masked later (past the end of the run) and only have to exist
+    uint2* lut = reinterpret_cast<uint2*>(smem + G_::LUT_OFF);
+    for (int i = threadIdx.x; i < kLutEntries; i += kWarps * 32) {
+        const uint32_t s2 = (i <= 255 ? pow2_f16(i - 255 + kTopShift) : 0u) * 0x00010001u;
+        lut[i] = make_uint2(s2, mul_f16x2(s2, kBias));
+    }
+    // integer score path: 2^(e - 129), the true weight of a mantissa unit, as fp32 (no range issue there)
+    float* lutf = reinterpret_cast<float*>(smem + G_::LUTF_OFF);
+    if (KI)
+        for (int i = threadIdx.x; i < 256; i += kWarps * 32) lutf[i] = unit_weight(i, 4);
+    __syncthreads();
+    if (i0 >= i1) return;
+
     // per-lane byte offsets inside a stage
     const int k_off = G_::KM_OFF + g * ROW_M + t * (KI ? 4 : 16);
     const int kei_off = G_::KE_OFF + g * ROW_E;
@@ -437,10 +449,6 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
         if (cr.n_tok == 0) continue;
 
         // ---- run set-up: exponent references, query fragments, score factors ------------------
-        const int dk = KI ? 0 : warp_max_byte(a.k_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
-        const int dv = warp_max_byte(a.v_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
-        const uint2* lutk = lut + (255 - dk);
-        const uint2* lutv = lut + (255 - dv);
         uint2 qf[NT][8];                  // fp16 path: B fragments of the coefficients
         float kfac[NT];
         uint32_t qi8[NT][8];              // integer path: B fragments of the coefficient digits
@@ -472,9 +480,22 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                         qf[nt][2 * j] = make_uint2(v.x, v.y);
                         qf[nt][2 * j + 1] = make_uint2(v.z, v.w);
                     }
-                    kfac[nt] = pow2_split(a.scale_log2e, dk - 129 - kTopShift + (qn < Gq ? meta[0] : 0));
+                    kfac[nt] = (float)(qn < Gq ? meta[0] : 0);      // the query's exponent; completed below
                 }
             }
+        }
+        // (after the fragment loads were issued, so that the two latencies overlap)
+        const int dk = KI ? 0 : warp_max_byte(a.k_exp + cr.row0 * ROW_E, cr.n_tok * ROW_E, lane);
+        const uint2* lutk = lut + (255 - dk);
+        // The V side finds its reference exponent on the way: every tile is checked against the current one
+        // before it is used, and the reference is raised (the accumulators scaled down by the exact power of
+        // two) when a tile holds a larger exponent byte.  The first tile of a run always raises it.
+        int dv = 0;
+        uint32_t dv_probe = 0x7FFF7FFFu;          // (0x7FFF - dv) in both halves: adding a byte > dv sets bit 15
+        const uint2* lutv = lut + 255;
+        if (!KI) {
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt) kfac[nt] = pow2_split(a.scale_log2e, dk - 129 - kTopShift + (int)kfac[nt]);
         }
         float o[NT][8][4];
 #pragma unroll
@@ -487,9 +508,56 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) { m_run[nt] = -INFINITY; l_run[nt] = 0.f; }
 
+        constexpr int VE_WORDS = kTile * ROW_E / 4;      // V exponent bytes of a stage, in words
+        // slow path of the check: largest V exponent byte among the tile's live rows; raise the reference to it
+        // (plus some headroom, so that small upward steps do not come back here)
+        auto raise_dv = [&](const uint8_t* st, int n_live) {
+            const int n_bytes = min(n_live, kTile) * ROW_E;
+            uint32_t m = 0;
+            for (int w = lane; w < VE_WORDS; w += 32) {
+                uint32_t x = *reinterpret_cast<const uint32_t*>(st + G_::VE_OFF + 4 * w);
+                const int left = n_bytes - 4 * w;
+                if (left < 4) x = left <= 0 ? 0u : (x & ((1u << (8 * left)) - 1u));
+                m = vmaxu4(m, x);
+            }
+#pragma unroll
+            for (int off = 16; off; off >>= 1) m = vmaxu4(m, __shfl_xor_sync(0xffffffffu, m, off));
+            m = vmaxu4(m, m >> 16);
+            m = vmaxu4(m, m >> 8);
+            const int dt = (int)(m & 0xffu);
+            if (dt > dv) {
+                const int nd = min(dt + kDvHeadroom, 255);
+                const float f = pow2_split(1.f, dv - nd);       // exact; underflows to 0 only with the sums it scales
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int r = 0; r < 8; ++r)
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) o[nt][r][k] *= f;
+                dv = nd;
+                dv_probe = (0x7FFFu - (uint32_t)nd) * 0x00010001u;
+                lutv = lut + (255 - nd);
+            }
+        };
+
         // one stage of kTile tokens; FULL = every row of the tile exists
         auto tile_body = [&](const uint8_t* st, int n_live, auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;
+            // ---- V exponent bytes against the reference: even and odd bytes in 16-bit lanes, bit 15 = "larger"
+            if (FULL) {
+                uint32_t f = 0;
+#pragma unroll
+                for (int i = 0; i < (VE_WORDS + 31) / 32; ++i) {
+                    const int w = lane + 32 * i;
+                    if (VE_WORDS % 32 == 0 || w < VE_WORDS) {
+                        const uint32_t x = *reinterpret_cast<const uint32_t*>(st + G_::VE_OFF + 4 * w);
+                        f |= ((x & 0x00FF00FFu) + dv_probe) | (prmt(x, 0u, 0x4341u) + dv_probe);
+                    }
+                }
+                if (__any_sync(0xffffffffu, (f & 0x80008000u) != 0u)) raise_dv(st, n_live);
+            } else {
+                raise_dv(st, n_live);         // rows past the end may hold anything: masked there
+            }
             // ---- scores ---------------------------------------------------------
             float sc[kMT][NT][2];
 #pragma unroll
