@@ -16,7 +16,7 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
                                                  const int32_t* __restrict__ inv_perm_v, float* __restrict__ out,
                                                  int n_rows, int n_q_heads, int group, int n_chunks, int chunk,
                                                  int len_cap, int n_warps, int item_tokens, int items_per_pair,
-                                                 long long n_items) {
+                                                 int range_items, int range_extra) {
     constexpr int D = kHeadDim;
     __shared__ float so[4][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -27,7 +27,7 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
     len = len < 0 ? 0 : (len > len_cap ? len_cap : len);
     const int nc = (len + item_tokens - 1) / item_tokens;        // items that hold tokens
     const float* base = partials + (int64_t)row * n_chunks * kPartStride;
-    const long long first = ((long long)b * (n_q_heads / group) + hq / group) * items_per_pair;   // first item of the pair
+    const int first = (b * (n_q_heads / group) + hq / group) * items_per_pair;   // first item of the pair
     float m = -INFINITY, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int i = 0; i < nc;) {
@@ -42,9 +42,8 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
                 if (n_warps == 0) {
                     ++i;
                 } else {                             // next partial of the pair: where the next range starts
-                    const long long item = first + i;
-                    const long long w = ((item + 1) * n_warps - 1) / n_items;      // range that holds this item
-                    i = (int)(((w + 1) * n_items) / n_warps - first);
+                    const int w = range_of(first + i, range_items, range_extra);    // range that holds this item
+                    i = range_start(w + 1, range_items, range_extra) - first;
                 }
             }
         }
@@ -188,8 +187,7 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
     const int n_rows = f.batch * n_q_heads;
     lse_merge<<<(n_rows + 3) / 4, 128, 0, s>>>(a.partials, seq_lens, inv_perm_v, out, n_rows, n_q_heads, group,
                                               a.n_chunks, a.chunk, a.len_cap, split.n_warps, split.item_tokens,
-                                              split.items_per_pair,
-                                              (long long)f.batch * f.n_kv_heads * split.items_per_pair);
+                                              split.items_per_pair, split.range_items, split.range_extra);
     KVBFP_LAUNCH_CHECK("lse_merge");
     return KVBFP_OK;
 }

@@ -28,6 +28,8 @@ struct DecodeArgs {
     int len_cap;              // min(max_len_hint, max_seq)
     int item_tokens;          // persistent kernel: tokens per work item (divides chunk) and items per (batch, kv head)
     int items_per_pair;
+    int range_items;          // persistent kernel: items of a warp's range; the first `range_extra` ranges hold one more
+    int range_extra;
     uint32_t* status;
     // 2^(32-k): multiplying by these and keeping the high word is a right shift by k that runs on the
     // multiply-add pipe instead of the integer pipe (passed at run time so that it stays a multiply)
@@ -37,13 +39,24 @@ struct DecodeArgs {
 kvbfp_status launch_decode_simt(const DecodeArgs& a, cudaStream_t s);
 kvbfp_status launch_decode_mma(const DecodeArgs& a, cudaStream_t s);    // bf16, every mantissa width
 // How the persistent kernel cut the work, for the merge: the items (pair-major pieces of `item_tokens` tokens,
-// `items_per_pair` per (batch, kv head)) were split into `n_warps` contiguous ranges.  n_warps == 0: no ranges,
+// `items_per_pair` per (batch, kv head)) were split into `n_warps` contiguous ranges of `range_items` items, the
+// first `range_extra` of them one item longer.  n_warps == 0: no ranges,
 // every chunk has its own partial.
 struct Split {
     int n_warps = 0;
     int item_tokens = 0;
     int items_per_pair = 0;
+    int range_items = 0;      // range w starts at item  w * range_items + min(w, range_extra)
+    int range_extra = 0;
 };
+// First item of range w, and the range that holds item x (32-bit: the launcher refuses 2^31 items and more).
+__host__ __device__ __forceinline__ int range_start(int w, int range_items, int range_extra) {
+    return w * range_items + (w < range_extra ? w : range_extra);
+}
+__host__ __device__ __forceinline__ int range_of(int x, int range_items, int range_extra) {
+    const int big = range_extra * (range_items + 1);             // items held by the longer ranges
+    return x < big ? x / (range_items + 1) : range_extra + (x - big) / range_items;
+}
 // Slot (chunk-sized, n_chunks per pair) that receives the partial of a run whose first item within its pair
 // is `item`.  Items are whole chunks, or half chunks: then two runs can start in the first chunk of a pair (one
 // that holds only item 0, the next from item 1 on), so odd items round up; ranges hold four items or more, so

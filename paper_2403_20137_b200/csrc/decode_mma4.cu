@@ -187,7 +187,8 @@ __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t*
 // every block are cast to C = round(c * 2^(14 - qe)) with the block's own exponent qe and written as two signed
 // byte digits, C = 256 * d1 + d0, in the B-fragment order of the byte MMA: fragment m = 2 * seg + kind covers the
 // bytes [16 seg, 16 seg + 16) of a row; lane (g, t) holds bytes 4t..4t+3 for column g = (query g/2, digit g%2:
-// 0 = d1, 1 = d0).  qmeta[query][2 blk] = qe, qmeta[query][2 blk + 1] = 136 * sum(C of kind 1) + 128 * sum(C of kind 2).
+// 0 = d1, 1 = d0).  qmeta[query][2 blk] = scale * log2(e) * 2^(qe - 14) as float bits,
+// qmeta[query][2 blk + 1] = 136 * sum(C of kind 1) + 128 * sum(C of kind 2).
 __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
     // one thread per slot, the four query heads of the n-tile in turn
     const int N = a.fmt.block, nblk = D / N;
@@ -246,7 +247,7 @@ __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_
         sC[qq][s] = C;
         atomicAdd(&sbias[qq][blk], ((s & 1) ? 136 : 128) * C);
         if (s % N == 0 && 4 * nt + qq < G)
-            qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * blk] = qe;
+            qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * blk] = __float_as_int(pow2_split(a.scale_log2e, qe - 14));
     }
     __syncthreads();
     if (s < 4 * nblk) {
@@ -348,17 +349,16 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
-    const int64_t n_items = (int64_t)a.fmt.batch * Hkv * a.items_per_pair;
-    const int64_t wglob = (int64_t)blockIdx.x * kWarps + warp, wtot = (int64_t)gridDim.x * kWarps;
-    const int64_t i0 = wglob * n_items / wtot, i1 = (wglob + 1) * n_items / wtot;     // this warp's items
-    auto get_run = [&](int64_t it) -> Run {
+    const int wglob = blockIdx.x * kWarps + warp;
+    const int i0 = range_start(wglob, a.range_items, a.range_extra);                  // this warp's items
+    const int i1 = i0 + a.range_items + (wglob < a.range_extra ? 1 : 0);
+    auto get_run = [&](int it) -> Run {
         Run r;
-        const int64_t pair = it / a.items_per_pair;
-        r.chunk0 = (int)(it - pair * a.items_per_pair);
-        r.hk = (int)(pair % Hkv);
-        r.b = (int)(pair / Hkv);
-        const int64_t left = i1 - it;
-        r.n_items = (int)(left < (int64_t)(a.items_per_pair - r.chunk0) ? left : (int64_t)(a.items_per_pair - r.chunk0));
+        const int pair = it / a.items_per_pair;
+        r.chunk0 = it - pair * a.items_per_pair;
+        r.b = pair / Hkv;
+        r.hk = pair - r.b * Hkv;
+        r.n_items = min(i1 - it, a.items_per_pair - r.chunk0);
         int len = a.seq_lens[r.b];
         if (len > a.fmt.max_seq || len < 0) {
             if (lane == 0 && r.chunk0 == 0 && r.hk == 0) raise_flag(a.status, KVBFP_FLAG_POSITION);
@@ -372,7 +372,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
         const int64_t tok1 = (int64_t)(r.chunk0 + r.n_items) * a.item_tokens;
         r.n_tok = max(0, (int)min((int64_t)len, tok1) - tok0);
         r.n_tiles = (r.n_tok + kTile - 1) / kTile;
-        r.row0 = pair * a.fmt.max_seq + tok0;
+        r.row0 = (int64_t)pair * a.fmt.max_seq + tok0;
         return r;
     };
 
@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
     const uint8_t* my_base = lane == 0 ? a.k_mant : lane == 1 ? a.v_mant : lane == 2 ? a.k_exp : a.v_exp;
     const int my_row_bytes = (lane < 2) ? ROW_M : ROW_E;
     const uint32_t my_dst = wsm_u32 + (lane == 0 ? G_::KM_OFF : lane == 1 ? G_::VM_OFF : lane == 2 ? G_::KE_OFF : G_::VE_OFF);
-    int64_t p_next = i0;
+    int p_next = i0;
     Run pr;
     pr.n_tiles = 0;
     int p_tile = 0;
@@ -443,7 +443,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
     uint32_t parity = 0;
     bool timed_out = false;
 
-    for (int64_t c_next = i0; c_next < i1 && !timed_out;) {
+    for (int c_next = i0; c_next < i1 && !timed_out;) {
         const Run cr = get_run(c_next);
         c_next += cr.n_items;
         if (cr.n_tok == 0) continue;
@@ -469,7 +469,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(Deco
                     }
 #pragma unroll
                     for (int k = 0; k < NBLK; ++k) {
-                        qfac[nt][k] = pow2_split(a.scale_log2e, meta[2 * k] - 14);
+                        qfac[nt][k] = __int_as_float(meta[2 * k]);
                         qbias[nt][k] = meta[2 * k + 1];
                     }
                 } else {
@@ -828,11 +828,14 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     b.item_tokens = fine ? kTile : a.chunk;
     b.items_per_pair = fine ? fine_per_pair : a.n_chunks;
     const int64_t n_items = pairs * b.items_per_pair;
+    if (n_items >= (int64_t)1 << 31) return KVBFP_ERR_UNSUPPORTED;         // item indices are 32-bit in the kernels
     const int64_t want = (n_items + kWarps - 1) / kWarps;
     const int grid = (int)(want < resident[dev] ? want : resident[dev]);
     split->n_warps = grid * kWarps;
     split->item_tokens = b.item_tokens;
     split->items_per_pair = b.items_per_pair;
+    b.range_items = split->range_items = (int)(n_items / split->n_warps);
+    b.range_extra = split->range_extra = (int)(n_items % split->n_warps);
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));

@@ -209,9 +209,11 @@ def rel_err(got, ref):
 
 
 def run_decode_case(oracle, w, Bn, S, lens, block, p, impl, use_perm=True, perm_v=False, max_seq=None,
-                    chunk_tokens=0, q_mant_bits=0, scale=0.0, hint=0):
+                    chunk_tokens=0, q_mant_bits=0, scale=0.0, hint=0, v_token_log2=None):
     max_seq = max_seq or ((S + 15) // 16) * 16
     k, v = W.make_kv(w, n_tokens=S, batch=Bn)
+    if v_token_log2 is not None:          # token t of V times 2^v_token_log2[t] (exact in bf16 and fp32)
+        v = (v.float() * torch.exp2(torch.as_tensor(v_token_log2, dtype=torch.float32)).view(1, S, 1, 1)).to(v.dtype)
     q = W.make_q(w, batch=Bn)
     pk = pv = ipv = None
     if use_perm:
@@ -293,6 +295,33 @@ def test_decode_split_invariance(oracle, impl):
         outs.append(got)
     for o in outs[1:]:
         assert rel_err(o, outs[0]) <= (1e-5 if impl == B.DECODE_SIMT else 1e-4)
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("n", [16, 32, 128])
+def test_decode_value_exponents_drift(oracle, impl, n):
+    """V magnitudes that climb and fall along the sequence, and that jump by 2^60 and up to the top of the
+    exponent range for a few tokens: the 4-bit kernel raises the reference exponent of its fp16 V weights
+    while it walks a run and rescales its sums, so every step of the way has to stay exact.  The softmax is
+    made nearly flat (small scale) so that every token carries weight and a wrong step shows in the result."""
+    w = W.CONFIGS[2]
+    S = 1500
+    t = np.arange(S)
+    flat = dict(scale=0.004)
+    climb = np.where(t < 750, t // 24, (1499 - t) // 24)               # +1 binade per 24 tokens, up to 2^31, and back
+    for chunk in (0, 1536):                                             # library's split; one run over all 24 stages
+        got, ref = run_decode_case(oracle, w, 1, S, [S], n, 4, impl, v_token_log2=climb, chunk_tokens=chunk, **flat)
+        assert np.isfinite(got).all() and rel_err(got, ref) <= ATTN_TOL
+    jump = np.zeros(S, dtype=np.int64)
+    jump[:200] = -20
+    jump[700:703] = 60
+    got, ref = run_decode_case(oracle, w, 1, S, [S], n, 4, impl, v_token_log2=jump, chunk_tokens=1536, **flat)
+    assert np.isfinite(got).all() and rel_err(got, ref) <= ATTN_TOL
+    # exponent bytes next to the largest one; the bf16 kernel's conversion (136 times the block's power of two
+    # as an intermediate) leaves the bf16 range above 2^120, which its header states as its limit
+    jump[1301] = 110 if impl == B.DECODE_MMA_BF16 else 122
+    got, ref = run_decode_case(oracle, w, 1, S, [S], n, 4, impl, v_token_log2=jump, **flat)
+    assert np.isfinite(got).all() and rel_err(got, ref) <= ATTN_TOL
 
 
 @pytest.mark.parametrize("impl", IMPLS)

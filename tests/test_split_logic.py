@@ -14,12 +14,24 @@ def partial_slot(item, item_tokens, chunk, n_chunks):
     return min((item + 1) >> 1, n_chunks - 1)
 
 
+def range_start(w, per, extra):
+    return w * per + min(w, extra)
+
+
+def range_of(x, per, extra):
+    big = extra * (per + 1)
+    return x // (per + 1) if x < big else extra + (x - big) // per
+
+
 def kernel_runs(pairs, ipp, W):
     """[(pair, first item in pair, n_items)] as the kernel's get_run() walks them."""
     n = pairs * ipp
+    per, extra = divmod(n, W)
     runs = []
     for w in range(W):
-        i0, i1 = w * n // W, (w + 1) * n // W
+        i0 = range_start(w, per, extra)
+        i1 = i0 + per + (1 if w < extra else 0)
+        assert i1 == range_start(w + 1, per, extra)
         it = i0
         while it < i1:
             pair, c0 = divmod(it, ipp)
@@ -31,12 +43,13 @@ def kernel_runs(pairs, ipp, W):
 
 def merge_heads(pair, ipp, W, n, nc):
     """First items of the runs of `pair` as lse_merge enumerates them (items < nc hold tokens)."""
+    per, extra = divmod(n, W)
     first, heads, i = pair * ipp, [], 0
     while i < nc:
         heads.append(i)
-        item = first + i
-        w = ((item + 1) * W - 1) // n
-        i = ((w + 1) * n) // W - first
+        w = range_of(first + i, per, extra)
+        assert range_start(w, per, extra) <= first + i < range_start(w + 1, per, extra)
+        i = range_start(w + 1, per, extra) - first
     return heads
 
 
@@ -53,7 +66,6 @@ def test_runs_match_merge_and_slots_are_unique():
         cases.append((pairs, ipp, W, 64 if fine else 128, 128))
     for pairs, ipp, W, item_tokens, chunk in cases:
         n = pairs * ipp
-        W = min(W, n)
         n_chunks = (ipp * item_tokens + chunk - 1) // chunk
         runs = kernel_runs(pairs, ipp, W)
         assert sum(c for _, _, c in runs) == n
