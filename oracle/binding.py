@@ -55,6 +55,8 @@ def lib():
                                      C.c_int, C.c_void_p, C.c_void_p]
         L.oracle_decode_attn.argtypes = [C.c_void_p] * 6 + [C.c_int, C.c_int] + [C.c_void_p] * 3 + \
             [C.c_double, C.c_int, C.c_void_p]
+        L.oracle_decode_attn_rope.argtypes = [C.c_void_p] * 6 + [C.c_int, C.c_int] + [C.c_void_p] * 3 + \
+            [C.c_double] + [C.c_void_p] * 4
         L.oracle_rope_tables.restype = None
         L.oracle_rope_tables.argtypes = [C.c_int, C.c_double, C.c_int, C.c_void_p, C.c_void_p, C.c_void_p]
         L.oracle_rope_permute_tables.restype = None
@@ -194,6 +196,23 @@ def decode_attn(cache, q, q_dtype, n_q_heads, seq_lens, perm_k=None, inv_perm_v=
     _check(lib().oracle_decode_attn(C.byref(f), _p(cache.k_mant), _p(cache.k_exp), _p(cache.v_mant),
                                     _p(cache.v_exp), _p(qq), _DT[q_dtype], n_q_heads, _p(sl), _p(pk),
                                     _p(ipv), float(softmax_scale), int(q_mant_bits), _p(out)))
+    return out
+
+
+def decode_attn_rope(cache, q, q_dtype, n_q_heads, seq_lens, theta, partner, sign, perm_k=None, inv_perm_v=None,
+                     softmax_scale=0.0):
+    """Attention over a cache of pre-rotation keys; theta/partner/sign: [n_kv_heads * head_dim] in stored order."""
+    f = cache.fmt
+    qq = _as_input(q, q_dtype)
+    sl = _c(seq_lens, np.int32)
+    pk = None if perm_k is None else _c(perm_k, np.int32)
+    ipv = None if inv_perm_v is None else _c(inv_perm_v, np.int32)
+    th, pa, sg = _c(theta, np.float64), _c(partner, np.int32), _c(sign, np.float64)
+    assert th.size == pa.size == sg.size == f.n_kv_heads * f.head_dim
+    out = np.zeros((f.batch, n_q_heads, f.head_dim), dtype=np.float64)
+    _check(lib().oracle_decode_attn_rope(C.byref(f), _p(cache.k_mant), _p(cache.k_exp), _p(cache.v_mant),
+                                         _p(cache.v_exp), _p(qq), _DT[q_dtype], n_q_heads, _p(sl), _p(pk),
+                                         _p(ipv), float(softmax_scale), _p(th), _p(pa), _p(sg), _p(out)))
     return out
 
 

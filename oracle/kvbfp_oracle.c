@@ -251,11 +251,14 @@ int oracle_dequant(const oracle_format* f, const uint8_t* mant, const uint8_t* e
 
 /* ---------------------------------------------------------------- attention */
 
-int oracle_decode_attn(const oracle_format* f, const uint8_t* k_mant, const uint8_t* k_exp,
-                       const uint8_t* v_mant, const uint8_t* v_exp, const void* q, int q_dt,
-                       int n_q_heads, const int32_t* seq_lens, const int32_t* perm_k,
-                       const int32_t* inv_perm_v, double softmax_scale, int q_mant_bits,
-                       double* out) {
+/* Attention over the cache; theta != NULL: the dequantised key row of token t is rotated to position t
+ * (Eq. (4) with the tables of Algorithm 1 step 5, one set of d entries per KV head) before the product. */
+static int decode_attn_impl(const oracle_format* f, const uint8_t* k_mant, const uint8_t* k_exp,
+                            const uint8_t* v_mant, const uint8_t* v_exp, const void* q, int q_dt,
+                            int n_q_heads, const int32_t* seq_lens, const int32_t* perm_k,
+                            const int32_t* inv_perm_v, double softmax_scale, int q_mant_bits,
+                            const double* theta, const int32_t* partner, const double* sign,
+                            double* out) {
     if (!format_ok(f) || !k_mant || !k_exp || !v_mant || !v_exp || !q || !seq_lens || !out)
         return ORACLE_INVALID;
     if (n_q_heads < 1 || n_q_heads % f->n_kv_heads != 0) return ORACLE_INVALID;
@@ -267,6 +270,7 @@ int oracle_decode_attn(const oracle_format* f, const uint8_t* k_mant, const uint
     int* M = (int*)malloc((size_t)d * sizeof(int));
     double* qp = (double*)malloc((size_t)d * sizeof(double));
     double* krow = (double*)malloc((size_t)d * sizeof(double));
+    double* krot = (double*)malloc((size_t)d * sizeof(double));
     double* o = (double*)malloc((size_t)d * sizeof(double));
     for (int b = 0; b < f->batch && rc == ORACLE_OK; ++b) {
         const int len = seq_lens[b];
@@ -300,8 +304,14 @@ int oracle_decode_attn(const oracle_format* f, const uint8_t* k_mant, const uint
             double smax = -INFINITY;
             for (int t = 0; t < len; ++t) {
                 dequant_row(f, k_mant + (base + t) * (int64_t)row_m, k_exp + (base + t) * (int64_t)row_e, M, krow);
+                const double* kt = krow;
+                if (theta) {   /* Sec. III par. 2: the rotary embedding is applied after the read-back */
+                    oracle_rope_apply(d, (double)t, theta + (int64_t)g * d, partner + (int64_t)g * d,
+                                      sign + (int64_t)g * d, krow, krot);
+                    kt = krot;
+                }
                 double acc = 0.0;
-                for (int j = 0; j < d; ++j) acc += qp[j] * krow[j];
+                for (int j = 0; j < d; ++j) acc += qp[j] * kt[j];
                 s[t] = scale * acc;
                 if (s[t] > smax) smax = s[t];
             }
@@ -327,8 +337,28 @@ int oracle_decode_attn(const oracle_format* f, const uint8_t* k_mant, const uint
     free(M);
     free(qp);
     free(krow);
+    free(krot);
     free(o);
     return rc;
+}
+
+int oracle_decode_attn(const oracle_format* f, const uint8_t* k_mant, const uint8_t* k_exp,
+                       const uint8_t* v_mant, const uint8_t* v_exp, const void* q, int q_dt,
+                       int n_q_heads, const int32_t* seq_lens, const int32_t* perm_k,
+                       const int32_t* inv_perm_v, double softmax_scale, int q_mant_bits,
+                       double* out) {
+    return decode_attn_impl(f, k_mant, k_exp, v_mant, v_exp, q, q_dt, n_q_heads, seq_lens, perm_k,
+                            inv_perm_v, softmax_scale, q_mant_bits, NULL, NULL, NULL, out);
+}
+
+int oracle_decode_attn_rope(const oracle_format* f, const uint8_t* k_mant, const uint8_t* k_exp,
+                            const uint8_t* v_mant, const uint8_t* v_exp, const void* q, int q_dt,
+                            int n_q_heads, const int32_t* seq_lens, const int32_t* perm_k,
+                            const int32_t* inv_perm_v, double softmax_scale, const double* theta,
+                            const int32_t* partner, const double* sign, double* out) {
+    if (!theta || !partner || !sign) return ORACLE_INVALID;
+    return decode_attn_impl(f, k_mant, k_exp, v_mant, v_exp, q, q_dt, n_q_heads, seq_lens, perm_k,
+                            inv_perm_v, softmax_scale, 0, theta, partner, sign, out);
 }
 
 /* --------------------------------------------------------- rotary embedding */

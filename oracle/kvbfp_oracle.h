@@ -100,6 +100,16 @@ int oracle_decode_attn(const oracle_format* f, const uint8_t* k_mant, const uint
                        const int32_t* inv_perm_v, double softmax_scale, int q_mant_bits,
                        double* out);
 
+/* The same over a cache of keys stored BEFORE the rotary embedding (Sec. III par. 2: the embedding is applied
+ * to the keys after they are read back): the dequantised key row of token t is rotated to position t by
+ * Eq. (4), with tables in stored order (Algorithm 1 step 5; [n_kv_heads * head_dim] each), and then
+ * multiplied with pi(q).  q is taken as given: already rotated to its own position by the caller. */
+int oracle_decode_attn_rope(const oracle_format* f, const uint8_t* k_mant, const uint8_t* k_exp,
+                            const uint8_t* v_mant, const uint8_t* v_exp, const void* q, int q_dt,
+                            int n_q_heads, const int32_t* seq_lens, const int32_t* perm_k,
+                            const int32_t* inv_perm_v, double softmax_scale, const double* theta,
+                            const int32_t* partner, const double* sign, double* out);
+
 /* Eq. (4): rotary embedding of x[d] at position m, in place.
  * theta[d], partner[d] (0-based index of the element whose value is taken for
  * the sine term) and sign[d] describe the layout; Algorithm 1 step 5 permutes

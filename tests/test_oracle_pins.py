@@ -495,6 +495,68 @@ def test_permuted_rope_commutes_with_permutation(oracle, half_split):
     assert abs(a - b) < 1e-12
 
 
+def _tables(oracle, perm, half_split):
+    """Per-head tables in stored order, concatenated [H * d]."""
+    H, d = perm.shape
+    theta, partner, sign = oracle.rope_tables(d, 10000.0, half_split)
+    out = [oracle.rope_permute_tables(perm[h], np.argsort(perm[h]).astype(np.int32), theta, partner, sign)
+           for h in range(H)]
+    return (np.concatenate([o[0] for o in out]), np.concatenate([o[1] for o in out]).astype(np.int32),
+            np.concatenate([o[2] for o in out]))
+
+
+@pytest.mark.parametrize("half_split", [False, True])
+def test_attention_over_pre_rotation_keys(oracle, half_split):
+    """Attention with the rotary embedding applied after the read-back (Sec. III par. 2), pinned to things other
+    than itself: (1) zero frequencies are no rotation at all; (2) the textbook form, complex multiplication of the
+    channel pairs by e^{i t theta}, on the dequantised keys with numpy's softmax; (3) with one block per row
+    (so that the cast does not depend on the order, Table I's last row) a K-sorted cache with the permuted tables
+    of Algorithm 1 step 5 gives what the unsorted cache gives with the plain tables."""
+    B, T, Hkv, Hq, d = 2, 37, 2, 4, 128
+    rng = np.random.default_rng(21)
+    k = (rng.standard_normal((B, T, Hkv, d)) * 2).astype(np.float32)
+    v = rng.standard_normal((B, T, Hkv, d)).astype(np.float32)
+    q = rng.standard_normal((B, Hq, d)).astype(np.float32)
+    lens = [37, 9]
+    ident = np.tile(np.arange(d, dtype=np.int32), (Hkv, 1))
+    th, pa, sg = _tables(oracle, ident, half_split)
+    c = oracle.Cache(B, Hkv, d, 48, 32, 4)
+    oracle.append(c, k, v, "f32", np.zeros(B, dtype=np.int32))
+    # (1)
+    plain = oracle.decode_attn(c, q, "f32", Hq, lens)
+    assert np.array_equal(oracle.decode_attn_rope(c, q, "f32", Hq, lens, np.zeros_like(th), pa, sg), plain)
+    # (2)
+    out = oracle.decode_attn_rope(c, q, "f32", Hq, lens, th, pa, sg)
+    assert not np.allclose(out, plain, rtol=1e-3)
+    freq = 10000.0 ** (-2.0 * np.arange(d // 2) / d)
+    for b in range(B):
+        for hq in range(Hq):
+            g = hq // (Hq // Hkv)
+            Kd = oracle.dequant(c, "k", b, g, 0, lens[b])
+            Vd = oracle.dequant(c, "v", b, g, 0, lens[b])
+            lo, hi = (Kd[:, :d // 2], Kd[:, d // 2:]) if half_split else (Kd[:, 0::2], Kd[:, 1::2])
+            z = (lo + 1j * hi) * np.exp(1j * np.arange(lens[b])[:, None] * freq[None, :])
+            Kr = np.empty_like(Kd)
+            if half_split:
+                Kr[:, :d // 2], Kr[:, d // 2:] = z.real, z.imag
+            else:
+                Kr[:, 0::2], Kr[:, 1::2] = z.real, z.imag
+            s = Kr @ q[b, hq].astype(np.float64) / math.sqrt(d)
+            pr = np.exp(s - s.max())
+            pr /= pr.sum()
+            assert np.allclose(out[b, hq], pr @ Vd, rtol=1e-11, atol=1e-12)
+    # (3)
+    perm = np.stack([rng.permutation(d) for _ in range(Hkv)]).astype(np.int32)
+    tp, pp, sp = _tables(oracle, perm, half_split)
+    c1 = oracle.Cache(B, Hkv, d, 48, 128, 4)
+    c2 = oracle.Cache(B, Hkv, d, 48, 128, 4)
+    oracle.append(c1, k, v, "f32", np.zeros(B, dtype=np.int32))
+    oracle.append(c2, k, v, "f32", np.zeros(B, dtype=np.int32), perm)
+    a = oracle.decode_attn_rope(c1, q, "f32", Hq, lens, th, pa, sg)
+    bb = oracle.decode_attn_rope(c2, q, "f32", Hq, lens, tp, pp, sp, perm_k=perm)
+    assert np.allclose(a, bb, rtol=1e-11, atol=1e-12)
+
+
 # ---------------------------------------------------------------- inputs follow the stated recipe
 def test_workload_recipe():
     w = W.CONFIGS[2]
