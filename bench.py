@@ -271,6 +271,8 @@ def main():
     ap.add_argument("--mant-bits", type=int, default=0, choices=[0, 4, 6, 8])
     ap.add_argument("--block", type=int, default=0, choices=[0, 16, 32, 64, 128])
     ap.add_argument("--chunk", type=int, default=0, help="tokens per sequence chunk (0 = library default)")
+    ap.add_argument("--rope", action="store_true", help="keys cached before the rotary embedding: time "
+                    "kvbfp_decode_attn_rope (fp32 kernel, rotation after the read-back) instead; no end-to-end leg")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the set-up timings and the quality report")
     ap.add_argument("--sweep5", action="store_true", help="add the prefill/append and calibration sweep (8 KV heads, 65536 new\n                    tokens, blocks 16/32/64 x mantissas 4/6/8, calibration over 2^20 tokens) to the extras")
@@ -307,7 +309,10 @@ def main():
     es = 2 if w.dtype == "bf16" else 4
     extras = {}
     calib = W.make_calibration(w, device=dev)
-    _, perm_k, _ = B.calibrate(calib, Hkv, d)
+    _, perm_k, inv_perm_k = B.calibrate(calib, Hkv, d)
+    if args.rope:
+        impl, kernel, args.no_e2e = B.DECODE_SIMT, "decode_simt_rope", True
+        rope_tabs = B.rope_tables(perm_k, inv_perm_k, Hkv, d, 10000.0, False, device=dev)
     if not args.no_extras:
         ms = timed(lambda: B.calibrate(calib, Hkv, d), reps=3)
         extras["calibrate"] = {"tokens": int(calib.shape[0]), "ms": ms, "GB/s": calib.numel() * es / ms / 1e6}
@@ -355,8 +360,11 @@ def main():
 
     def step():
         B.append(cache, k_new, v_new, start_pos, perm_k=perm_k)
-        B.decode_attn(cache, q, seq_lens, perm_k=perm_k, max_len_hint=S, impl=impl, out=out, workspace=ws,
-                      chunk_tokens=args.chunk)
+        if args.rope:
+            B.decode_attn_rope(cache, q, seq_lens, *rope_tabs, perm_k=perm_k, max_len_hint=S, out=out, workspace=ws)
+        else:
+            B.decode_attn(cache, q, seq_lens, perm_k=perm_k, max_len_hint=S, impl=impl, out=out, workspace=ws,
+                          chunk_tokens=args.chunk)
 
     def barrier():
         if dist is not None:

@@ -216,6 +216,26 @@ kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* q, kvbfp_dt
                                void* stream);
 
 /*
+ * kvbfp_decode_attn over a cache whose keys were stored BEFORE the rotary embedding (Sec. III par. 2: the
+ * embedding is applied to the keys after they are read back from the cache; Sec. II-D, Eq. (4); tables in
+ * stored order per Algorithm 1 step 5).  Token t's dequantised key row is rotated to position t, in registers,
+ * before the product with pi(q):  k'[j] = k[j] cos(t theta_j) + sign_j k[partner_j] sin(t theta_j).
+ *   q                    as in kvbfp_decode_attn, already rotated to its own position by the caller
+ *   theta, partner, sign [n_kv_heads*head_dim] f64 / i32 / f32 as written by kvbfp_rope_tables for the
+ *                        permutation the keys were appended with (partners share a frequency and have
+ *                        opposite signs; other tables give unspecified results)
+ *   flags                KVBFP_DECODE_AUTO or KVBFP_DECODE_SIMT (the fp32 kernel is the only one that rotates:
+ *                        KVBFP_ERR_UNSUPPORTED otherwise); chunks are capped at 512 tokens
+ * Everything else (workspace, lengths, V side, merge, errors) as in kvbfp_decode_attn.  No BFP query cast.
+ */
+kvbfp_status kvbfp_decode_attn_rope(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt,
+                                    int32_t n_q_heads, const int32_t* seq_lens, int32_t max_len_hint,
+                                    const int32_t* perm_k, const int32_t* inv_perm_v, float softmax_scale,
+                                    const double* theta, const int32_t* partner, const float* sign,
+                                    float* out, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                    void* stream);
+
+/*
  * kvbfp_decode_attn for callers that must not allocate device memory (the paper has no counterpart:
  * this is a deployment aid, not a step of the method).  Who needs it: code that runs after a serving
  * process has frozen its memory pool, plug-ins that are handed tensors but no allocator, and loops

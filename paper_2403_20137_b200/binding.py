@@ -24,7 +24,7 @@ EXPORTS = ["kvbfp_version", "kvbfp_status_string", "kvbfp_last_cuda_error", "kvb
            "kvbfp_decode_workspace_bytes", "kvbfp_decode_attn", "kvbfp_device_status",
            "kvbfp_launch_count", "kvbfp_step_staging_bytes", "kvbfp_decode_step_host",
            "kvbfp_profile_decode_events", "kvbfp_static_scratch_bytes", "kvbfp_decode_attn_static",
-           "kvbfp_rope_tables", "kvbfp_rope_apply"]
+           "kvbfp_rope_tables", "kvbfp_rope_apply", "kvbfp_decode_attn_rope"]
 
 
 class KvbfpError(RuntimeError):
@@ -97,6 +97,9 @@ def lib():
         L.kvbfp_decode_attn_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int32,
                                                C.c_void_p, C.c_void_p, C.c_float, C.c_int32, C.c_void_p,
                                                C.c_uint32, C.c_void_p]
+        L.kvbfp_decode_attn_rope.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int32, C.c_void_p, C.c_int32,
+                                             C.c_void_p, C.c_void_p, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_size_t, C.c_uint32, C.c_void_p]
         L.kvbfp_rope_tables.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_double, C.c_int32,
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.kvbfp_rope_apply.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
@@ -237,6 +240,27 @@ def decode_attn(cache, q, seq_lens, perm_k=None, inv_perm_v=None, softmax_scale=
                                    _ptr(_dev(inv_perm_v, torch.int32)), float(softmax_scale), q_mant_bits,
                                    _ptr(_dev(out, torch.float32)), _ptr(workspace), workspace.numel(), flags,
                                    _stream(stream)))
+    return out
+
+
+def decode_attn_rope(cache, q, seq_lens, theta, partner, sign, perm_k=None, inv_perm_v=None, softmax_scale=0.0,
+                     max_len_hint=0, impl=DECODE_AUTO, chunk_tokens=0, out=None, workspace=None, stream=None):
+    """kvbfp_decode_attn_rope: as decode_attn over keys cached before the rotary embedding; theta (f64), partner
+    (i32), sign (f32) are the [H_kv, d] tables of rope_tables()."""
+    q = _dev(q)
+    n_q_heads = q.shape[1]
+    if out is None:
+        out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = torch.empty(decode_workspace_bytes(cache.fmt, n_q_heads), dtype=torch.uint8, device=q.device)
+    flags = impl | ((chunk_tokens // 128) << 8)
+    cs = cache.struct()
+    _check(lib().kvbfp_decode_attn_rope(C.byref(cs), _ptr(q), _dt(q), n_q_heads, _ptr(_dev(seq_lens, torch.int32)),
+                                        max_len_hint, _ptr(_dev(perm_k, torch.int32)),
+                                        _ptr(_dev(inv_perm_v, torch.int32)), float(softmax_scale),
+                                        _ptr(_dev(theta, torch.float64)), _ptr(_dev(partner, torch.int32)),
+                                        _ptr(_dev(sign, torch.float32)), _ptr(_dev(out, torch.float32)),
+                                        _ptr(workspace), workspace.numel(), flags, _stream(stream)))
     return out
 
 

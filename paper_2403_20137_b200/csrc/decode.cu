@@ -112,12 +112,15 @@ extern "C" size_t kvbfp_decode_workspace_bytes(const kvbfp_format* fmt, int32_t 
     return qfrag_bytes(*fmt, n_q_heads) + part;
 }
 
-extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt,
-                                          int32_t n_q_heads, const int32_t* seq_lens, int32_t max_len_hint,
-                                          const int32_t* perm_k, const int32_t* inv_perm_v, float softmax_scale,
-                                          int32_t q_mant_bits, float* out, void* workspace, size_t workspace_bytes,
-                                          uint32_t flags, void* stream) {
-    using namespace kvbfp;
+namespace kvbfp {
+namespace {
+// The decode entry points: argument checks, chunking, main kernel, merge.  rope_theta != nullptr: keys are rotated
+// to their positions after the read-back (fp32 kernel).
+kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt, int32_t n_q_heads,
+                           const int32_t* seq_lens, int32_t max_len_hint, const int32_t* perm_k,
+                           const int32_t* inv_perm_v, float softmax_scale, int32_t q_mant_bits,
+                           const double* rope_theta, const int32_t* rope_partner, const float* rope_sign,
+                           float* out, void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
     if (!cache) return KVBFP_ERR_INVALID_ARG;
     const kvbfp_format& f = cache->fmt;
     kvbfp_status st = check_format(&f);
@@ -130,9 +133,16 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
     if (q_dt != KVBFP_F32 && q_dt != KVBFP_BF16) return KVBFP_ERR_INVALID_ARG;
     if (q_mant_bits != 0 && q_mant_bits != 8) return KVBFP_ERR_UNSUPPORTED;
     if (max_len_hint < 0 || !(softmax_scale >= 0.f) || isinf(softmax_scale)) return KVBFP_ERR_INVALID_ARG;
-    const uint32_t impl = flags & 0xffu, chunk_units = (flags >> 8) & 0xfffu;
+    uint32_t impl = flags & 0xffu, chunk_units = (flags >> 8) & 0xfffu;
     if (impl > KVBFP_DECODE_MMA_BF16 || (flags >> 20)) return KVBFP_ERR_INVALID_ARG;
-    const void* ptrs[] = {cache->k_mant, cache->k_exp, cache->v_mant, cache->v_exp, q, out, workspace, perm_k, inv_perm_v};
+    if (rope_theta) {
+        if (impl != KVBFP_DECODE_AUTO && impl != KVBFP_DECODE_SIMT) return KVBFP_ERR_UNSUPPORTED;
+        impl = KVBFP_DECODE_SIMT;
+        // the rotation is carried from token to token in fp32: short chunks keep that chain short
+        if (chunk_units == 0 || chunk_units > 4) chunk_units = 4;
+    }
+    const void* ptrs[] = {cache->k_mant, cache->k_exp, cache->v_mant, cache->v_exp, q, out, workspace, perm_k, inv_perm_v,
+                          rope_theta, rope_partner, rope_sign};
     for (const void* p : ptrs)
         if (p && !aligned16(p)) return KVBFP_ERR_ALIGNMENT;
     const size_t need = kvbfp_decode_workspace_bytes(&f, n_q_heads);
@@ -146,6 +156,7 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)f.head_dim);
     a.scale_log2e = scale * 1.4426950408889634f;
     a.q_mant_bits = q_mant_bits;
+    a.rope_theta = rope_theta; a.rope_partner = rope_partner; a.rope_sign = rope_sign;
     a.out = out;
     a.qfrag = static_cast<uint32_t*>(workspace);
     a.partials = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + qfrag_bytes(f, n_q_heads));
@@ -190,6 +201,28 @@ extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* 
                                               split.items_per_pair, split.range_items, split.range_extra);
     KVBFP_LAUNCH_CHECK("lse_merge");
     return KVBFP_OK;
+}
+}  // namespace
+}  // namespace kvbfp
+
+extern "C" kvbfp_status kvbfp_decode_attn(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt,
+                                          int32_t n_q_heads, const int32_t* seq_lens, int32_t max_len_hint,
+                                          const int32_t* perm_k, const int32_t* inv_perm_v, float softmax_scale,
+                                          int32_t q_mant_bits, float* out, void* workspace, size_t workspace_bytes,
+                                          uint32_t flags, void* stream) {
+    return kvbfp::decode_common(cache, q, q_dt, n_q_heads, seq_lens, max_len_hint, perm_k, inv_perm_v, softmax_scale,
+                                q_mant_bits, nullptr, nullptr, nullptr, out, workspace, workspace_bytes, flags, stream);
+}
+
+extern "C" kvbfp_status kvbfp_decode_attn_rope(const kvbfp_cache* cache, const void* q, kvbfp_dtype q_dt,
+                                               int32_t n_q_heads, const int32_t* seq_lens, int32_t max_len_hint,
+                                               const int32_t* perm_k, const int32_t* inv_perm_v, float softmax_scale,
+                                               const double* theta, const int32_t* partner, const float* sign,
+                                               float* out, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                               void* stream) {
+    if (!theta || !partner || !sign) return KVBFP_ERR_INVALID_ARG;
+    return kvbfp::decode_common(cache, q, q_dt, n_q_heads, seq_lens, max_len_hint, perm_k, inv_perm_v, softmax_scale, 0,
+                                theta, partner, sign, out, workspace, workspace_bytes, flags, stream);
 }
 
 extern "C" kvbfp_status kvbfp_profile_decode_events(void* start_event, void* stop_event) {

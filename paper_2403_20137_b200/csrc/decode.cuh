@@ -30,6 +30,10 @@ struct DecodeArgs {
     int items_per_pair;
     int range_items;          // persistent kernel: items of a warp's range; the first `range_extra` ranges hold one more
     int range_extra;
+    // keys cached before the rotary embedding (fp32 kernel only): tables in stored order, [n_kv_heads * head_dim]
+    const double* rope_theta;
+    const int32_t* rope_partner;
+    const float* rope_sign;
     uint32_t* status;
     // 2^(32-k): multiplying by these and keeping the high word is a right shift by k that runs on the
     // multiply-add pipe instead of the integer pipe (passed at run time so that it stays a multiply)

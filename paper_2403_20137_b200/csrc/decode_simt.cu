@@ -44,7 +44,18 @@ __device__ __forceinline__ float slot_value(const uint32_t (&w)[P], int i) {
     return (float)((int)(v & ((1u << P) - 1u)) - (1 << (P - 1)));
 }
 
-template <int P, int N>
+// cos and sin of an angle given in fp64 (token position times frequency, up to ~1e6 rad): reduced to [-pi, pi]
+// in fp64, evaluated in fp32.
+__device__ __forceinline__ void sincos_reduced(double angle, float* sn, float* cs) {
+    const double k = rint(angle * 0.15915494309189535);                        // 1 / (2 pi)
+    const double r = fma(-k, 2.4492935982947064e-16, fma(-k, 6.283185307179586, angle));   // 2 pi in two terms
+    sincosf((float)r, sn, cs);
+}
+
+// ROPE: the cache holds keys as they were before the rotary embedding (Sec. III par. 2); the rotation of
+// token t's key to position t is moved onto the query: q . R_t k = (R_t^T q) . k, and R_t^T q is carried from
+// token to token by a fixed rotation (the lane's tokens are 8 apart).
+template <int P, int N, bool ROPE>
 __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
     constexpr int D = kHeadDim, ROW_M = D * P / 8, ROW_E = D / N;
     constexpr int NB = (N == 16) ? 2 : 1;          // blocks inside one lane's 32 slots
@@ -104,6 +115,30 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
 #pragma unroll
         for (int i = 0; i < 32; ++i) q[i] *= a.scale_log2e;
     }
+    // ROPE state of slot i for the lane's current token t:  q[i] = q_i cos(t th_i) + q'_i sin(t th_i)  (the
+    // coefficient of k_i in the score), qw[i] = q'_i cos - q_i sin, with q'_i = -sign_i q_partner(i) (Eq. (4),
+    // partners share a frequency and have opposite signs); c8, s8 = cos, sin of 8 th_i advance both by 8 tokens.
+    float qw[ROPE ? 32 : 1], c8[ROPE ? 32 : 1], s8[ROPE ? 32 : 1];
+    if (ROPE) {
+        const int64_t qbase = ((int64_t)b * a.n_q_heads + hq) * D;
+        const double pos0 = (double)(t0 + r);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int slot = g * D + 32 * c + i;
+            const int pj = a.rope_partner[slot] & (D - 1);
+            const int ch = a.perm_k ? (a.perm_k[g * D + pj] & (D - 1)) : pj;
+            const float qp = (a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[qbase + ch])
+                                          : static_cast<const float*>(a.q)[qbase + ch]) * a.scale_log2e;
+            const float q1 = -a.rope_sign[slot] * qp;
+            const double th = a.rope_theta[slot];
+            float sn, cs;
+            sincos_reduced(pos0 * th, &sn, &cs);
+            const float q0 = q[i];
+            q[i] = q0 * cs + q1 * sn;
+            qw[i] = q1 * cs - q0 * sn;
+            sincos_reduced(8.0 * th, &s8[i], &c8[i]);
+        }
+    }
 
     const int64_t row0 = ((int64_t)b * Hkv + g) * a.fmt.max_seq;
     const uint8_t* km = a.k_mant + row0 * ROW_M + c * (4 * P);
@@ -130,6 +165,14 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
 #pragma unroll
                 for (int i = blk * (32 / NB); i < (blk + 1) * (32 / NB); ++i) acc = fmaf(q[i], slot_value<P>(w, i), acc);
                 s = fmaf(acc, unit_weight(ke[(int64_t)tok * ROW_E + eb + blk], P), s);
+            }
+        }
+        if (ROPE) {       // on to the lane's next token, 8 further
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float u = q[i], w = qw[i];
+                q[i] = fmaf(u, c8[i], w * s8[i]);
+                qw[i] = fmaf(w, c8[i], -u * s8[i]);
             }
         }
         s += __shfl_xor_sync(0xffffffffu, s, 1);
@@ -179,26 +222,36 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
     }
 }
 
-template <int P, int N>
+template <int P, int N, bool ROPE>
 kvbfp_status launch(const DecodeArgs& a, cudaStream_t s) {
     const int64_t n_items = (int64_t)a.fmt.batch * a.n_q_heads * a.n_chunks;
     const int grid = (int)((n_items + kWarps - 1) / kWarps);
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_simt<P, N><<<grid, kWarps * 32, 0, s>>>(a);
+    decode_simt<P, N, ROPE><<<grid, kWarps * 32, 0, s>>>(a);
     KVBFP_LAUNCH_CHECK("decode_simt");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;
 }
 
-template <int P>
+template <int P, bool ROPE>
 kvbfp_status launch_n(const DecodeArgs& a, cudaStream_t s) {
     switch (a.fmt.block) {
-        case 16: return launch<P, 16>(a, s);
-        case 32: return launch<P, 32>(a, s);
-        case 64: return launch<P, 64>(a, s);
-        case 128: return launch<P, 128>(a, s);
+        case 16: return launch<P, 16, ROPE>(a, s);
+        case 32: return launch<P, 32, ROPE>(a, s);
+        case 64: return launch<P, 64, ROPE>(a, s);
+        case 128: return launch<P, 128, ROPE>(a, s);
+    }
+    return KVBFP_ERR_UNSUPPORTED;
+}
+
+template <bool ROPE>
+kvbfp_status launch_p(const DecodeArgs& a, cudaStream_t s) {
+    switch (a.fmt.mant_bits) {
+        case 4: return launch_n<4, ROPE>(a, s);
+        case 6: return launch_n<6, ROPE>(a, s);
+        case 8: return launch_n<8, ROPE>(a, s);
     }
     return KVBFP_ERR_UNSUPPORTED;
 }
@@ -206,12 +259,7 @@ kvbfp_status launch_n(const DecodeArgs& a, cudaStream_t s) {
 }  // namespace
 
 kvbfp_status launch_decode_simt(const DecodeArgs& a, cudaStream_t s) {
-    switch (a.fmt.mant_bits) {
-        case 4: return launch_n<4>(a, s);
-        case 6: return launch_n<6>(a, s);
-        case 8: return launch_n<8>(a, s);
-    }
-    return KVBFP_ERR_UNSUPPORTED;
+    return a.rope_theta ? launch_p<true>(a, s) : launch_p<false>(a, s);
 }
 
 }  // namespace kvbfp

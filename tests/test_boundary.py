@@ -88,6 +88,11 @@ def test_host_side_argument_errors():
     assert L.kvbfp_decode_attn(*args(qb=4)) == B.ERR_UNSUPPORTED
     assert L.kvbfp_decode_attn(*args(flags=4)) == B.ERR_INVALID_ARG
     assert L.kvbfp_decode_attn(*args(scale=-1.0)) == B.ERR_INVALID_ARG
+    rope = lambda **k: [C.byref(cs), vp(16), 0, 4, vp(16), 0, None, None, 0.0, k.get("th", vp(16)), vp(16), vp(16), vp(16),
+                        vp(16), need, k.get("flags", 0), None]
+    assert L.kvbfp_decode_attn_rope(*rope(th=None)) == B.ERR_INVALID_ARG
+    assert L.kvbfp_decode_attn_rope(*rope(th=vp(8))) == B.ERR_ALIGNMENT
+    assert L.kvbfp_decode_attn_rope(*rope(flags=2)) == B.ERR_UNSUPPORTED    # tensor-core kernels do not rotate
     assert L.kvbfp_rope_tables(vp(16), None, 1, 128, 10000.0, 0, vp(16), vp(16), vp(16), None) == B.ERR_INVALID_ARG
     assert L.kvbfp_rope_tables(None, None, 1, 64, 10000.0, 0, vp(16), vp(16), vp(16), None) == B.ERR_UNSUPPORTED
     assert L.kvbfp_rope_apply(vp(16), 0, 4, 1, 128, vp(16), vp(16), vp(16), vp(16), vp(16), None) == B.ERR_INVALID_ARG   # y == x

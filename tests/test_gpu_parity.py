@@ -402,6 +402,39 @@ def test_rope_tables_and_apply(oracle, half_split):
 
 
 # ------------------------------------------------------------------------------- full-size workloads
+@pytest.mark.parametrize("half_split", [False, True])
+@pytest.mark.parametrize("p,n", [(4, 32), (4, 16), (8, 128), (6, 64)])
+def test_decode_over_pre_rotation_keys(oracle, half_split, p, n):
+    """Keys cached before the rotary embedding and K-sorted; the kernel rotates token t's key to position t after
+    the read-back (Sec. III par. 2) with the tables of Algorithm 1 step 5.  GQA, ragged lengths over several
+    chunks, positions up to 2999."""
+    import dataclasses
+    w = dataclasses.replace(W.CONFIGS[4], n_q_heads=8, n_kv_heads=2)
+    Bn, S, d, Hkv, Hq = 2, 3000, 128, 2, 8
+    lens = [3000, 517]
+    k, v = W.make_kv(w, n_tokens=S, batch=Bn)
+    q = W.make_q(w, batch=Bn)
+    _, pk, ipk = oracle.calibrate(W.to_oracle(k.reshape(-1, Hkv, d)), w.dtype, Hkv, d)
+    theta, partner, sign = oracle.rope_tables(d, 10000.0, half_split)
+    tabs = [oracle.rope_permute_tables(pk[h], ipk[h], theta, partner, sign) for h in range(Hkv)]
+    th, pa, sg = (np.concatenate([t[i] for t in tabs]) for i in range(3))
+    oc = oracle_cache(oracle, k, v, w.dtype, n, p, S + 8, perm_k=pk)
+    ref = oracle.decode_attn_rope(oc, W.to_oracle(q), w.dtype, Hq, lens, th, pa.astype(np.int32), sg, perm_k=pk)
+    plain = oracle.decode_attn(oc, W.to_oracle(q), w.dtype, Hq, lens, perm_k=pk)
+    assert rel_err(plain, ref) > 0.05                       # the rotation matters on this input
+    t = lambda a: dev(torch.from_numpy(np.ascontiguousarray(a)))
+    gth, gpa, gsg = B.rope_tables(t(pk), t(ipk), Hkv, d, 10000.0, half_split)
+    assert np.allclose(host(gth).ravel(), th, rtol=1e-14, atol=0) and np.array_equal(host(gpa).ravel(), pa)
+    gc = B.Cache(Bn, Hkv, d, S + 8, n, p, fill=0xFF)
+    B.append(gc, dev(k), dev(v), dev(torch.zeros(Bn, dtype=torch.int32)), t(pk))
+    out = B.decode_attn_rope(gc, dev(q), dev(torch.tensor(lens, dtype=torch.int32)), gth, gpa, gsg, perm_k=t(pk))
+    assert B.device_status() == 0
+    assert rel_err(host(out).astype(np.float64), ref) <= ATTN_TOL
+    with pytest.raises(B.KvbfpError):                       # only the fp32 kernel rotates
+        B.decode_attn_rope(gc, dev(q), dev(torch.tensor(lens, dtype=torch.int32)), gth, gpa, gsg, perm_k=t(pk),
+                           impl=B.DECODE_MMA)
+
+
 def _full_size_case(oracle, cfg, sample_pairs):
     """The benchmark's own launch (full batch, full sequence, library-chosen chunking) with inputs drawn on
     the GPU; the oracle recomputes sampled (batch, kv head) units one by one from the same raw inputs."""
