@@ -304,7 +304,8 @@ def main():
     # ---- set-up (untimed for the step metric): calibrate, prefill S-1 tokens ----------------------
     impl = {"auto": B.DECODE_AUTO, "simt": B.DECODE_SIMT, "mma": B.DECODE_MMA, "mma_bf16": B.DECODE_MMA_BF16}[args.decode_impl]
     kernel = "decode_simt" if impl == B.DECODE_SIMT else \
-        ("decode_mma4" if (w.mant_bits == 4 and impl != B.DECODE_MMA_BF16) else "decode_mma")
+        ("decode_mma4" if (w.mant_bits == 4 and impl != B.DECODE_MMA_BF16) else
+         "decode_mma8" if (w.mant_bits == 8 and w.block >= 32 and impl != B.DECODE_MMA_BF16) else "decode_mma")
     S, Bn, Hkv, Hq, d = w.seq, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim
     es = 2 if w.dtype == "bf16" else 4
     extras = {}
@@ -439,7 +440,7 @@ def main():
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16" if kernel == "decode_mma4" else ("bf16" if kernel == "decode_mma" else "f32"),
+        "dtype": "f16" if kernel in ("decode_mma4", "decode_mma8") else ("bf16" if kernel == "decode_mma" else "f32"),
         "data": "synthetic",
         "config": {"workload": workload_name(w), "per_gpu_batch": Bn, "decode_kernel": kernel,
                    "l2": f"inputs larger than L2: {alg / 1e6:.0f} MB of cache read per step vs 126 MB L2",

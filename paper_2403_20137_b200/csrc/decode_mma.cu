@@ -16,6 +16,11 @@
 // Output: O^T[16 slots x 8 cols] += V^T[16 slots x 16 tokens] . P^T[16 tokens x 8 cols], with the
 // softmax weights split into hi/lo halves the same way.  Accumulators are fp32.
 //
+// Range.  The bias product (136, 160 or 2304 units of the block's weight for 4-, 6- and 8-bit mantissas) is a bf16
+// intermediate of about 2^5 times the block's largest value, so cache values of magnitude 2^120 and above are
+// outside this kernel's range (they give infinities); the fp32 kernel and the 4- and 8-bit integer-score kernels
+// have no such limit.
+//
 // The integer pipe (logic ops, shifts, byte permutes) is what limits this kernel: every field is
 // extracted with one three-input logic instruction and block weights come from a 256-entry table in
 // shared memory instead of being rebuilt from the exponent byte.  (Issuing shifts as multiply-high on

@@ -298,11 +298,11 @@ def test_decode_split_invariance(oracle, impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("n", [16, 32, 128])
-def test_decode_value_exponents_drift(oracle, impl, n):
+@pytest.mark.parametrize("p,n", [(4, 16), (4, 32), (4, 128), (8, 32), (8, 64)])
+def test_decode_value_exponents_drift(oracle, impl, p, n):
     """V magnitudes that climb and fall along the sequence, and that jump by 2^60 and up to the top of the
-    exponent range for a few tokens: the 4-bit kernel raises the reference exponent of its fp16 V weights
-    while it walks a run and rescales its sums, so every step of the way has to stay exact.  The softmax is
+    exponent range for a few tokens: the 4-bit and 8-bit kernels raise the reference exponent of their fp16 V weights
+    while they walk a run and rescale their sums, so every step of the way has to stay exact.  The softmax is
     made nearly flat (small scale) so that every token carries weight and a wrong step shows in the result."""
     w = W.CONFIGS[2]
     S = 1500
@@ -310,17 +310,17 @@ def test_decode_value_exponents_drift(oracle, impl, n):
     flat = dict(scale=0.004)
     climb = np.where(t < 750, t // 24, (1499 - t) // 24)               # +1 binade per 24 tokens, up to 2^31, and back
     for chunk in (0, 1536):                                             # library's split; one run over all 24 stages
-        got, ref = run_decode_case(oracle, w, 1, S, [S], n, 4, impl, v_token_log2=climb, chunk_tokens=chunk, **flat)
+        got, ref = run_decode_case(oracle, w, 1, S, [S], n, p, impl, v_token_log2=climb, chunk_tokens=chunk, **flat)
         assert np.isfinite(got).all() and rel_err(got, ref) <= ATTN_TOL
     jump = np.zeros(S, dtype=np.int64)
     jump[:200] = -20
     jump[700:703] = 60
-    got, ref = run_decode_case(oracle, w, 1, S, [S], n, 4, impl, v_token_log2=jump, chunk_tokens=1536, **flat)
+    got, ref = run_decode_case(oracle, w, 1, S, [S], n, p, impl, v_token_log2=jump, chunk_tokens=1536, **flat)
     assert np.isfinite(got).all() and rel_err(got, ref) <= ATTN_TOL
     # exponent bytes next to the largest one; the bf16 kernel's conversion (136 times the block's power of two
     # as an intermediate) leaves the bf16 range above 2^120, which its header states as its limit
     jump[1301] = 110 if impl == B.DECODE_MMA_BF16 else 122
-    got, ref = run_decode_case(oracle, w, 1, S, [S], n, 4, impl, v_token_log2=jump, **flat)
+    got, ref = run_decode_case(oracle, w, 1, S, [S], n, p, impl, v_token_log2=jump, **flat)
     assert np.isfinite(got).all() and rel_err(got, ref) <= ATTN_TOL
 
 
