@@ -70,6 +70,40 @@ __host__ __device__ __forceinline__ int partial_slot(int item, int item_tokens, 
     const int s = (item + 1) >> 1;
     return s < n_chunks ? s : n_chunks - 1;
 }
+// Work split of a persistent kernel (host side).  Items are pieces of `fine_tokens` tokens (half a chunk) when the
+// library chose the chunking (chunk == kMinChunk == 2 * fine_tokens) and every warp still gets five or more of them
+// on average, so four at the least (the ranges then differ by one piece of work at most and partial_slot() keeps
+// the runs' partial results apart); whole chunks otherwise.  The items are cut into one contiguous range per warp
+// of min(capacity, blocks needed) thread blocks.  Fills the range fields of `b` and `split`, returns the grid.
+inline kvbfp_status plan_persistent(const DecodeArgs& a, int fine_tokens, int capacity_blocks, int warps_per_block,
+                                    DecodeArgs* b, Split* split, int* grid) {
+    *b = a;
+    const int64_t pairs = (int64_t)a.fmt.batch * a.fmt.n_kv_heads;
+    const int fine_per_pair = (a.len_cap + fine_tokens - 1) / fine_tokens;
+    const bool fine = a.chunk == 2 * fine_tokens && a.chunk == kMinChunk &&
+                      pairs * fine_per_pair >= 5LL * capacity_blocks * warps_per_block;
+    b->item_tokens = fine ? fine_tokens : a.chunk;
+    b->items_per_pair = fine ? fine_per_pair : a.n_chunks;
+    const int64_t n_items = pairs * b->items_per_pair;
+    if (n_items >= (int64_t)1 << 31) return KVBFP_ERR_UNSUPPORTED;         // item indices are 32-bit in the kernels
+    const int64_t want = (n_items + warps_per_block - 1) / warps_per_block;
+    *grid = (int)(want < capacity_blocks ? want : capacity_blocks);
+    split->n_warps = *grid * warps_per_block;
+    split->item_tokens = b->item_tokens;
+    split->items_per_pair = b->items_per_pair;
+    b->range_items = split->range_items = (int)(n_items / split->n_warps);
+    b->range_extra = split->range_extra = (int)(n_items % split->n_warps);
+    return KVBFP_OK;
+}
+// The items of one (batch, kv head) that fall into a warp's item range (persistent kernels).
+struct Run {
+    int b, hk;
+    int chunk0;        // first item within the pair: the slot of the chunk it lies in receives the partial result
+    int n_items;       // items covered (>= 1)
+    int n_tok;         // tokens that exist in them (0: nothing to do)
+    int n_tiles;
+    int64_t row0;      // first row in the planes
+};
 // 4-bit mantissas: integer scores + fp16 P.V, persistent
 kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, Split* split);
 // 8-bit mantissas, blocks of 32 slots or more: integer scores on the stored bytes + fp16 P.V, persistent

@@ -79,19 +79,6 @@ constexpr int kLutEntries = 512;        // index = exponent byte - D + 255, D = 
 constexpr uint32_t kMagic = 0x64646464u;        // 0x64 = high byte of fp16 1024.0
 constexpr uint32_t kBias = 0xE488E488u;         // fp16 -1160.0 twice
 
-// fp16 bit pattern of 2^j for j in [-24, 15], 0 below.
-__device__ __forceinline__ uint32_t pow2_f16(int j) {
-    if (j >= -14) return (uint32_t)(j + 15) << 10;
-    if (j >= -24) return 1u << (j + 24);
-    return 0u;
-}
-
-// 2^ex as a float for any ex that the product with an ordinary number keeps in range (two exact factors).
-__device__ __forceinline__ float pow2_split(float x, int ex) {
-    const int e1 = ex / 2, e2 = ex - e1;
-    return (x * exp2f((float)e1)) * exp2f((float)e2);
-}
-
 // Byte `byte` (0..63) of a row: low nibble = slot 2*byte, high nibble = slot 2*byte+1.
 // K side, k position kk (0..3 = k 2t, 2t+1, 2t+8, 2t+9) of k-step ks for lane column t:
 //   byte = 16t + 4(ks/2) + 2(ks%2) + (kk%2), kind 1 (whole byte) for kk < 2, kind 2 (low nibble) for kk >= 2.
@@ -327,16 +314,6 @@ __device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int la
     m = vmaxu4(m, m >> 8);
     return (int)(m & 0xffu);
 }
-
-// The chunks of one (batch, kv head) that fall into a warp's item range.
-struct Run {
-    int b, hk;
-    int chunk0;        // first item within the pair: the slot of the chunk it lies in receives the partial result
-    int n_items;       // items covered (>= 1)
-    int n_tok;         // tokens that exist in them (0: nothing to do)
-    int n_tiles;
-    int64_t row0;      // first row in the planes
-};
 
 template <int N, int NT>
 __global__ void __launch_bounds__(kWarps * 32, KVBFP4_MIN_CTAS) decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta) {
@@ -818,24 +795,10 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     if (N >= 32) make_qfrag4i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
     else make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
     KVBFP_LAUNCH_CHECK("make_qfrag4");
-    // Work items: one stage (kTile tokens) each when the library chose the chunking and every warp still gets
-    // at least four of them (half chunks: the ranges then differ by one stage of work at most; partial_slot()
-    // keeps the runs' partial results apart); whole chunks otherwise.
-    DecodeArgs b = a;
-    const int64_t pairs = (int64_t)a.fmt.batch * a.fmt.n_kv_heads;
-    const int fine_per_pair = (a.len_cap + kTile - 1) / kTile;
-    const bool fine = a.chunk == 2 * kTile && a.chunk == kMinChunk && pairs * fine_per_pair >= 4LL * resident[dev] * kWarps;
-    b.item_tokens = fine ? kTile : a.chunk;
-    b.items_per_pair = fine ? fine_per_pair : a.n_chunks;
-    const int64_t n_items = pairs * b.items_per_pair;
-    if (n_items >= (int64_t)1 << 31) return KVBFP_ERR_UNSUPPORTED;         // item indices are 32-bit in the kernels
-    const int64_t want = (n_items + kWarps - 1) / kWarps;
-    const int grid = (int)(want < resident[dev] ? want : resident[dev]);
-    split->n_warps = grid * kWarps;
-    split->item_tokens = b.item_tokens;
-    split->items_per_pair = b.items_per_pair;
-    b.range_items = split->range_items = (int)(n_items / split->n_warps);
-    b.range_extra = split->range_extra = (int)(n_items % split->n_warps);
+    DecodeArgs b;
+    int grid = 0;
+    const kvbfp_status st = plan_persistent(a, kTile, resident[dev], kWarps, &b, split, &grid);
+    if (st != KVBFP_OK) return st;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));

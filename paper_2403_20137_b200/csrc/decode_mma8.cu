@@ -40,16 +40,6 @@ constexpr int kLutEntries = 512;
 constexpr uint32_t kMagic = 0x64646464u;        // 0x64 = high byte of fp16 1024.0
 constexpr uint32_t kBias = 0xE480E480u;         // fp16 -1152.0 twice
 
-__device__ __forceinline__ uint32_t pow2_f16(int j) {      // fp16 bits of 2^j for j in [-24, 15], 0 below
-    if (j >= -14) return (uint32_t)(j + 15) << 10;
-    if (j >= -24) return 1u << (j + 24);
-    return 0u;
-}
-__device__ __forceinline__ float pow2_split(float x, int ex) {      // x * 2^ex in two exact factors
-    const int e1 = ex / 2, e2 = ex - e1;
-    return (x * exp2f((float)e1)) * exp2f((float)e2);
-}
-
 // ------------------------------------------------------------------ query fragments
 // One 128-thread block per (batch, kv head, n-tile of four query heads); thread s = slot s.  Fragment m (0..7) of an
 // n-tile covers row bytes {32 (m/2) + 8 t + 4 (m%2) + e : t, e = 0..3}: lane (g, t) of the main kernel reads eight
@@ -144,15 +134,6 @@ struct Geo8 {
     static constexpr int LUTF_OFF = LUT_OFF + kLutEntries * 8;          // float[256]
     static constexpr int BAR_OFF = LUTF_OFF + 256 * 4;
     static constexpr int SMEM_BYTES = BAR_OFF + kWarps * kStages * 8;
-};
-
-struct Run {
-    int b, hk;
-    int chunk0;        // first item within the pair
-    int n_items;
-    int n_tok;         // tokens that exist in them (0: nothing to do)
-    int n_tiles;
-    int64_t row0;      // first row in the planes
 };
 
 template <int N, int NT>
@@ -543,23 +524,10 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
     make_qfrag8i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
     KVBFP_LAUNCH_CHECK("make_qfrag8i");
-    // Work items: half chunks when the library chose the chunking and every warp still gets five or more of them
-    // (partial_slot() keeps the runs' partial results apart); whole chunks otherwise.
-    DecodeArgs b = a;
-    const int64_t pairs = (int64_t)a.fmt.batch * a.fmt.n_kv_heads;
-    const int fine_per_pair = (a.len_cap + kItemFine - 1) / kItemFine;
-    const bool fine = a.chunk == 2 * kItemFine && a.chunk == kMinChunk && pairs * fine_per_pair >= 5LL * resident[dev] * kWarps;
-    b.item_tokens = fine ? kItemFine : a.chunk;
-    b.items_per_pair = fine ? fine_per_pair : a.n_chunks;
-    const int64_t n_items = pairs * b.items_per_pair;
-    if (n_items >= (int64_t)1 << 31) return KVBFP_ERR_UNSUPPORTED;         // item indices are 32-bit in the kernels
-    const int64_t want = (n_items + kWarps - 1) / kWarps;
-    const int grid = (int)(want < resident[dev] ? want : resident[dev]);
-    split->n_warps = grid * kWarps;
-    split->item_tokens = b.item_tokens;
-    split->items_per_pair = b.items_per_pair;
-    b.range_items = split->range_items = (int)(n_items / split->n_warps);
-    b.range_extra = split->range_extra = (int)(n_items % split->n_warps);
+    DecodeArgs b;
+    int grid = 0;
+    const kvbfp_status st = plan_persistent(a, kItemFine, resident[dev], kWarps, &b, split, &grid);
+    if (st != KVBFP_OK) return st;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));

@@ -122,4 +122,16 @@ __device__ __forceinline__ void mma_u8s8_first(int (&d)[4], uint32_t a0, uint32_
 }
 __device__ __forceinline__ uint32_t vmaxu4(uint32_t a, uint32_t b) { return __vmaxu4(a, b); }
 
+// fp16 bit pattern of 2^j for j in [-24, 15], 0 below.
+__device__ __forceinline__ uint32_t pow2_f16(int j) {
+    if (j >= -14) return (uint32_t)(j + 15) << 10;
+    if (j >= -24) return 1u << (j + 24);
+    return 0u;
+}
+// x * 2^ex for any ex that keeps the product in range (two exact factors).
+__device__ __forceinline__ float pow2_split(float x, int ex) {
+    const int e1 = ex / 2, e2 = ex - e1;
+    return (x * exp2f((float)e1)) * exp2f((float)e2);
+}
+
 }  // namespace kvbfp
