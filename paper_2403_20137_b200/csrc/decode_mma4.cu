@@ -177,7 +177,8 @@ __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t*
 // 0 = d1, 1 = d0).  qmeta[query][2 blk] = scale * log2(e) * 2^(qe - 14) as float bits,
 // qmeta[query][2 blk + 1] = 136 * sum(C of kind 1) + 128 * sum(C of kind 2).
 __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
-    // one thread per slot, the four query heads of the n-tile in turn
+    // one thread per slot, the four query heads of the n-tile in turn; a block of 32 slots or more is made of whole
+    // warps, so block maxima and sums are reduced in the warp first
     const int N = a.fmt.block, nblk = D / N;
     const int s = threadIdx.x, blk = s / N;
     const int item = blockIdx.x;
@@ -201,7 +202,10 @@ __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_
     }
     if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
 #pragma unroll
-        for (int qq = 0; qq < 4; ++qq) atomicMax(&smax[0][qq][blk], __float_as_uint(v[qq]) & 0x7fffffffu);
+        for (int qq = 0; qq < 4; ++qq) {
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(v[qq]) & 0x7fffffffu);
+            if ((s & 31) == 0) atomicMax(&smax[0][qq][blk], mx);
+        }
         __syncthreads();
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) {
@@ -220,7 +224,8 @@ __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_
     for (int qq = 0; qq < 4; ++qq) {
         const float other = __shfl_xor_sync(0xffffffffu, v[qq], 1);
         c[qq] = (s & 1) ? v[qq] * 0.0625f : (v[qq] - other * 0.0625f) * 0.0625f;
-        atomicMax(&smax[1][qq][blk], __float_as_uint(c[qq]) & 0x7fffffffu);
+        const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(c[qq]) & 0x7fffffffu);
+        if ((s & 31) == 0) atomicMax(&smax[1][qq][blk], mx);
     }
     __syncthreads();
 #pragma unroll
@@ -232,7 +237,8 @@ __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_
         const int sh = 14 - qe, h1 = sh / 2, h2 = sh - h1;    // two exact factors (sh in [-114, 140])
         const int C = __float2int_rn((c[qq] * pow2i(h1)) * pow2i(h2));
         sC[qq][s] = C;
-        atomicAdd(&sbias[qq][blk], ((s & 1) ? 136 : 128) * C);
+        const int bsum = __reduce_add_sync(0xffffffffu, ((s & 1) ? 136 : 128) * C);
+        if ((s & 31) == 0) atomicAdd(&sbias[qq][blk], bsum);
         if (s % N == 0 && 4 * nt + qq < G)
             qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * blk] = __float_as_int(pow2_split(a.scale_log2e, qe - 14));
     }

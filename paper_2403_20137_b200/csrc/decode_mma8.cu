@@ -70,7 +70,10 @@ __global__ void __launch_bounds__(128) make_qfrag8i(DecodeArgs a, int NT, int32_
     }
     if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
 #pragma unroll
-        for (int qq = 0; qq < 4; ++qq) atomicMax(&smax[0][qq][blk], __float_as_uint(v[qq]) & 0x7fffffffu);
+        for (int qq = 0; qq < 4; ++qq) {
+            const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(v[qq]) & 0x7fffffffu);
+            if ((s & 31) == 0) atomicMax(&smax[0][qq][blk], mx);
+        }
         __syncthreads();
 #pragma unroll
         for (int qq = 0; qq < 4; ++qq) {
@@ -82,7 +85,10 @@ __global__ void __launch_bounds__(128) make_qfrag8i(DecodeArgs a, int NT, int32_
         }
     }
 #pragma unroll
-    for (int qq = 0; qq < 4; ++qq) atomicMax(&smax[1][qq][blk], __float_as_uint(v[qq]) & 0x7fffffffu);
+    for (int qq = 0; qq < 4; ++qq) {
+        const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(v[qq]) & 0x7fffffffu);
+        if ((s & 31) == 0) atomicMax(&smax[1][qq][blk], mx);
+    }
     __syncthreads();
 #pragma unroll
     for (int qq = 0; qq < 4; ++qq) {
@@ -93,7 +99,8 @@ __global__ void __launch_bounds__(128) make_qfrag8i(DecodeArgs a, int NT, int32_
         const int sh = 14 - qe, h1 = sh / 2, h2 = sh - h1;    // two exact factors
         const int C = __float2int_rn((v[qq] * pow2i(h1)) * pow2i(h2));
         sC[qq][s] = C;
-        atomicAdd(&sbias[qq][blk], 128 * C);
+        const int bsum = __reduce_add_sync(0xffffffffu, 128 * C);
+        if ((s & 31) == 0) atomicAdd(&sbias[qq][blk], bsum);
         if (s % N == 0 && 4 * nt + qq < G)
             qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * blk] = __float_as_int(pow2_split(a.scale_log2e, qe - 14));
     }
