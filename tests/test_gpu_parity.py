@@ -481,3 +481,40 @@ def test_full_size_config3_sampled(oracle):
 def test_full_size_config4_gqa_sampled(oracle):
     """B8, 32 query heads on 8 KV heads, S32768: two sampled (batch, kv head) units, four query heads each."""
     _full_size_case(oracle, 4, [(0, 0), (7, 5)])
+
+
+@pytest.mark.parametrize("p,impl", [(4, B.DECODE_AUTO), (8, B.DECODE_AUTO), (6, B.DECODE_AUTO), (4, B.DECODE_SIMT)])
+def test_planes_beyond_4_gib(oracle, p, impl):
+    """Maximum sizes: a cache whose mantissa planes are larger than 4 GiB (40 sequences x 32 heads x 65536 rows),
+    so that row offsets need 64 bits in append, dequant and decode.  300 tokens are written to every sequence;
+    the last sequence's units (byte offsets above 2^32) are compared with the oracle run on that sequence alone."""
+    w = W.CONFIGS[2]
+    Bn, Hkv, d, S_max, T, n = 40, 32, 128, 65536, 300, 32
+    dv = torch.device("cuda")
+    cache = B.Cache(Bn, Hkv, d, S_max, n, p, device=dv)
+    assert cache.k_mant.numel() > (1 << 32)
+    k, v = W.make_kv(w, n_tokens=T, device=dv, batch=Bn)
+    q = W.make_q(w, device=dv, batch=Bn)
+    start = torch.full((Bn,), 1000, dtype=torch.int32, device=dv)
+    B.append(cache, k, v, start)
+    lens = torch.zeros(Bn, dtype=torch.int32, device=dv)
+    lens[Bn - 1] = 1000 + T
+    lens[0] = 1000 + T
+    # rows [0, 1000) of the two sequences that are read: zeros as keys and values (written, so that they are specified)
+    zk = torch.zeros(Bn, 1000, Hkv, d, dtype=k.dtype, device=dv)
+    B.append(cache, zk, zk, torch.zeros(Bn, dtype=torch.int32, device=dv))
+    del zk
+    out = B.decode_attn(cache, q, lens, max_len_hint=1000 + T, impl=impl)
+    assert B.device_status() == 0
+    assert not host(out[1:Bn - 1]).any()                       # empty sequences
+    for b in (0, Bn - 1):
+        for h in (0, Hkv - 1):
+            kk = np.concatenate([np.zeros((1, 1000, 1, d), np.float32), host(k[b:b + 1, :, h:h + 1].float())], axis=1)
+            vv = np.concatenate([np.zeros((1, 1000, 1, d), np.float32), host(v[b:b + 1, :, h:h + 1].float())], axis=1)
+            oc = oracle.Cache(1, 1, d, 1312, n, p)
+            oracle.append(oc, kk, vv, "f32", np.zeros(1, np.int32))
+            assert np.array_equal(host(cache.k_mant[b, h, :1000 + T]), oc.k_mant[0, 0, :1000 + T])
+            assert np.array_equal(host(cache.v_exp[b, h, :1000 + T]), oc.v_exp[0, 0, :1000 + T])
+            assert np.array_equal(host(B.dequant(cache, "v", b, h, 1000, T)), oracle.dequant(oc, "v", 0, 0, 1000, T).astype(np.float32))
+            ref = oracle.decode_attn(oc, W.to_oracle(q[b:b + 1, h:h + 1]), w.dtype, 1, [1000 + T])
+            assert rel_err(host(out[b:b + 1, h:h + 1]).astype(np.float64), ref) <= ATTN_TOL
