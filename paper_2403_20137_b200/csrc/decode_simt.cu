@@ -152,19 +152,38 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
     for (int i = 0; i < 32; ++i) o[i] = 0.f;
     float m = -INFINITY, l = 0.f;
 
+    // The packed words and exponent bytes of the lane's next token are loaded before the current token is worked
+    // on: with a handful of warps per SM the kernel is otherwise bound by the latency of these loads.
+    struct Tok {
+        uint32_t k[P], v[P];
+        uint32_t ke[NB], ve[NB];
+    };
+    auto fetch = [&](int tok, Tok& x) {
+        if (tok < t1) {
+            load_chunk<P>(km + (int64_t)tok * ROW_M, x.k);
+            load_chunk<P>(vm + (int64_t)tok * ROW_M, x.v);
+#pragma unroll
+            for (int blk = 0; blk < NB; ++blk) {
+                x.ke[blk] = __ldg(ke + (int64_t)tok * ROW_E + eb + blk);
+                x.ve[blk] = __ldg(ve + (int64_t)tok * ROW_E + eb + blk);
+            }
+        }
+    };
+    Tok nxt;
+    fetch(t0 + r, nxt);
     for (int tb = t0; tb < t1; tb += 8) {
         const int tok = tb + r;
         const bool valid = tok < t1;
+        const Tok cur = nxt;
+        fetch(tok + 8, nxt);
         float s = 0.f;
         if (valid) {
-            uint32_t w[P];
-            load_chunk<P>(km + (int64_t)tok * ROW_M, w);
 #pragma unroll
             for (int blk = 0; blk < NB; ++blk) {
                 float acc = 0.f;
 #pragma unroll
-                for (int i = blk * (32 / NB); i < (blk + 1) * (32 / NB); ++i) acc = fmaf(q[i], slot_value<P>(w, i), acc);
-                s = fmaf(acc, unit_weight(ke[(int64_t)tok * ROW_E + eb + blk], P), s);
+                for (int i = blk * (32 / NB); i < (blk + 1) * (32 / NB); ++i) acc = fmaf(q[i], slot_value<P>(cur.k, i), acc);
+                s = fmaf(acc, unit_weight((int)cur.ke[blk], P), s);
             }
         }
         if (ROPE) {       // on to the lane's next token, 8 further
@@ -187,13 +206,11 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
             }
             const float p = exp2f(s - m);
             l += p;
-            uint32_t w[P];
-            load_chunk<P>(vm + (int64_t)tok * ROW_M, w);
 #pragma unroll
             for (int blk = 0; blk < NB; ++blk) {
-                const float pw = p * unit_weight(ve[(int64_t)tok * ROW_E + eb + blk], P);
+                const float pw = p * unit_weight((int)cur.ve[blk], P);
 #pragma unroll
-                for (int i = blk * (32 / NB); i < (blk + 1) * (32 / NB); ++i) o[i] = fmaf(pw, slot_value<P>(w, i), o[i]);
+                for (int i = blk * (32 / NB); i < (blk + 1) * (32 / NB); ++i) o[i] = fmaf(pw, slot_value<P>(cur.v, i), o[i]);
             }
         }
     }
