@@ -117,8 +117,12 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
     }
     // ROPE state of slot i for the lane's current token t:  q[i] = q_i cos(t th_i) + q'_i sin(t th_i)  (the
     // coefficient of k_i in the score), qw[i] = q'_i cos - q_i sin, with q'_i = -sign_i q_partner(i) (Eq. (4),
-    // partners share a frequency and have opposite signs); c8, s8 = cos, sin of 8 th_i advance both by 8 tokens.
-    float qw[ROPE ? 32 : 1], c8[ROPE ? 32 : 1], s8[ROPE ? 32 : 1];
+    // partners share a frequency and have opposite signs); cos and sin of 8 th_i advance both by 8 tokens.
+    // (the step rotation sits in shared memory, one (cos, sin) pair per slot and warp: it only depends on the head,
+    // and 64 more registers per lane would leave no room for the prefetched words)
+    float qw[ROPE ? 32 : 1];
+    __shared__ float2 step_cs[ROPE ? kWarps : 1][ROPE ? 32 * 4 : 1];
+    float2* my_cs = &step_cs[ROPE ? (threadIdx.x >> 5) : 0][0];
     if (ROPE) {
         const int64_t qbase = ((int64_t)b * a.n_q_heads + hq) * D;
         const double pos0 = (double)(t0 + r);
@@ -136,8 +140,13 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
             const float q0 = q[i];
             q[i] = q0 * cs + q1 * sn;
             qw[i] = q1 * cs - q0 * sn;
-            sincos_reduced(8.0 * th, &s8[i], &c8[i]);
+            if (r == 0) {       // the warp's eight token groups share the head, so one of them fills the table
+                float sn8, cs8;
+                sincos_reduced(8.0 * th, &sn8, &cs8);
+                my_cs[i * 4 + c] = make_float2(cs8, sn8);
+            }
         }
+        __syncwarp();
     }
 
     const int64_t row0 = ((int64_t)b * Hkv + g) * a.fmt.max_seq;
@@ -190,8 +199,9 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const float u = q[i], w = qw[i];
-                q[i] = fmaf(u, c8[i], w * s8[i]);
-                qw[i] = fmaf(w, c8[i], -u * s8[i]);
+                const float2 cs = my_cs[i * 4 + c];
+                q[i] = fmaf(u, cs.x, w * cs.y);
+                qw[i] = fmaf(w, cs.x, -u * cs.y);
             }
         }
         s += __shfl_xor_sync(0xffffffffu, s, 1);
