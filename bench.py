@@ -49,11 +49,13 @@ def sources_hash(kernel):
     return h.hexdigest()
 
 
-def traffic_per_launch(kernel, units):
+def traffic_per_launch(kernel, w):
+    """DRAM bytes of one launch, scaled from the capture by the units processed; None when there is no capture for
+    this kernel and format (the capture is of block 32, 4-bit mantissas) or the kernel has changed since."""
     t = TRAFFIC.get(kernel)
-    if not t or not t["bytes_per_unit"] or t["sources_sha256"] != sources_hash(kernel):
+    if not t or not t["bytes_per_unit"] or (w.block, w.mant_bits) != (32, 4) or t["sources_sha256"] != sources_hash(kernel):
         return None
-    return t["bytes_per_unit"] * units
+    return t["bytes_per_unit"] * decode_units(w)
 
 
 def workload_name(w):
@@ -450,7 +452,7 @@ def main():
                 "ms_per_step": (ms_e2e / args.steps) if n_e2e else None},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "traffic": traffic_per_launch(kernel, decode_units(w)),
+                     "frac": achieved / peak, "traffic": traffic_per_launch(kernel, w),
                      "algorithmic_bytes": alg, "kernel_ms": kernel_ms, "peak_source": peak_src},
         "extras": extras or None,
     }
