@@ -264,11 +264,12 @@ def test_decode_gqa(oracle, impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-def test_decode_group_of_8_and_2(oracle, impl):
+@pytest.mark.parametrize("p,n", [(4, 32), (8, 32), (8, 128), (6, 64)])
+def test_decode_group_of_8_and_2(oracle, impl, p, n):
     import dataclasses
     for hq, hkv in ((16, 2), (4, 2)):
         w = dataclasses.replace(W.CONFIGS[4], n_q_heads=hq, n_kv_heads=hkv)
-        got, ref = run_decode_case(oracle, w, 1, 150, [150], 32, 4, impl)
+        got, ref = run_decode_case(oracle, w, 1, 150, [150], n, p, impl)
         assert rel_err(got, ref) <= ATTN_TOL
 
 
@@ -281,7 +282,8 @@ def test_decode_empty_and_capacity_edges(oracle, impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-def test_decode_split_invariance(oracle, impl):
+@pytest.mark.parametrize("p", [4, 8])
+def test_decode_split_invariance(oracle, impl, p):
     """The chunk count must not matter: 1, 2, 7 and 52 chunks agree with each other.  The fp32 kernel
     agrees to 1e-5; the tensor-core kernel carries q and the softmax weights as two bf16 terms
     (2^-16 relative each), and a different chunking moves the softmax reference point, so its runs
@@ -290,7 +292,7 @@ def test_decode_split_invariance(oracle, impl):
     S = 6600
     outs = []
     for chunk in (6656, 3328, 1024, 128):
-        got, ref = run_decode_case(oracle, w, 1, S, [S], 32, 4, impl, chunk_tokens=chunk)
+        got, ref = run_decode_case(oracle, w, 1, S, [S], 32, p, impl, chunk_tokens=chunk)
         assert rel_err(got, ref) <= ATTN_TOL
         outs.append(got)
     for o in outs[1:]:
@@ -330,6 +332,8 @@ def test_decode_bfp16_query_and_scale(oracle, impl):
     got, ref = run_decode_case(oracle, w, 1, 300, [300], 32, 4, impl, q_mant_bits=8, scale=0.05)
     assert rel_err(got, ref) <= ATTN_TOL
     got, ref = run_decode_case(oracle, w, 1, 300, [300], 64, 4, impl, q_mant_bits=8)
+    assert rel_err(got, ref) <= ATTN_TOL
+    got, ref = run_decode_case(oracle, w, 1, 300, [300], 32, 8, impl, q_mant_bits=8, scale=0.05)   # 8-bit cache as well
     assert rel_err(got, ref) <= ATTN_TOL
 
 
