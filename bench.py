@@ -223,7 +223,16 @@ def sweep_config5(B, dev):
     _, perm, _ = B.calibrate(calib, H, d)
     ms = timed(lambda: B.calibrate(calib, H, d), reps=3)
     out["calibrate"] = {"tokens": int(calib.shape[0]), "ms": ms, "GB/s": calib.numel() * 2 / ms / 1e6}
-    del calib
+    # the paper's own front end: Euclidean norm of the rows of W_k (given transposed, [d_in, H*d]), rows folded by the
+    # permutation (Algorithm 1 steps 1, 3-4)
+    wk_t = calib[:4096]                                             # stands in for W_k^T: [4096, 8, 128]
+    _, perm_l2, _ = B.calibrate(wk_t, H, d, stat=B.STAT_L2)
+    ms = timed(lambda: B.calibrate(wk_t, H, d, stat=B.STAT_L2), reps=5)
+    out["calibrate_l2"] = {"rows": 4096, "ms": ms, "GB/s": wk_t.numel() * 2 / ms / 1e6}
+    wk = torch.randn(H * d, 4096, dtype=torch.bfloat16, device=dev, generator=torch.Generator(device=dev).manual_seed(7))
+    ms = timed(lambda: B.fold_perm(wk, perm_l2, H, d), reps=5)
+    out["fold_perm"] = {"shape": [H * d, 4096], "ms": ms, "GB/s": 2 * wk.numel() * 2 / ms / 1e6}
+    del calib, wk, wk_t
     k, v = W.make_kv(w, n_tokens=T, device=dev, batch=1)             # [1, 65536, 8, 128]
     z = torch.zeros(1, dtype=torch.int32, device=dev)
     ref = k[0, :4096, 0].float()
@@ -242,6 +251,18 @@ def sweep_config5(B, dev):
                                 "key_mse_unsorted": mse_u, "key_mse_ksort": mse_s}
             del c
     out["append"] = fm
+    # read-back paths on the last cache: dequantisation of one head, rotation of rows in stored order
+    c = B.Cache(1, H, d, T, 32, 4, device=dev)
+    B.append(c, k, v, z, perm_k=perm)
+    ms = timed(lambda: B.dequant(c, "k", 0, 0, 0, T, perm=perm), reps=5)
+    out["dequant_one_head"] = {"tokens": T, "ms": ms, "GB/s": T * (68 + d * 4) / ms / 1e6}
+    _, _, inv = B.calibrate(k[0, :4096].contiguous(), H, d)
+    tabs = B.rope_tables(perm, inv, H, d, 10000.0, False, device=dev)
+    rows = k[0]
+    pos = torch.arange(T, dtype=torch.int32, device=dev)
+    B.rope_apply(rows, pos, *tabs)
+    ms = timed(lambda: B.rope_apply(rows, pos, *tabs), reps=5)
+    out["rope_apply"] = {"rows": T * H, "ms": ms, "GB/s": 2 * rows.numel() * 2 / ms / 1e6}
     return out
 
 

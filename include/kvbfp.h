@@ -177,7 +177,7 @@ kvbfp_status kvbfp_rope_tables(const int32_t* perm, const int32_t* inv_perm, int
 
 /*
  * Eq. (4) in table form on rows in slot order: y[j] = x[j] cos(m theta_j) + sign_j x[partner_j] sin(m theta_j),
- * m = positions[row].  The angle is formed in fp64; y is rounded once to `dt`.
+ * m = positions[row].  The angle is formed and reduced in fp64, the rotation itself is fp32 (about 1e-7 relative).
  *   x, y       [n_rows, n_heads, head_dim] of `dt`, y != x
  *   positions  [n_rows] i32
  */

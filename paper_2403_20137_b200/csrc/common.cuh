@@ -60,6 +60,14 @@ __device__ __forceinline__ float unit_weight(int e8, int p) {
     return f >= 1 ? __uint_as_float((uint32_t)f << 23) : __uint_as_float(1u << (22 + f));
 }
 
+// cos and sin of an angle given in fp64 (token position times frequency, up to ~1e6 rad): reduced to [-pi, pi]
+// in fp64, evaluated in fp32.
+__device__ __forceinline__ void sincos_reduced(double angle, float* sn, float* cs) {
+    const double k = rint(angle * 0.15915494309189535);                        // 1 / (2 pi)
+    const double r = fma(-k, 2.4492935982947064e-16, fma(-k, 6.283185307179586, angle));   // 2 pi in two terms
+    sincosf((float)r, sn, cs);
+}
+
 __device__ __forceinline__ void raise_flag(uint32_t* status, uint32_t bit) { atomicOr(status, bit); }
 
 // Mantissa stored in the p-bit field (excess-2^(p-1) code) starting at bit `bit` of a little-endian byte row.

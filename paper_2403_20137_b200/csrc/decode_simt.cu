@@ -44,14 +44,6 @@ __device__ __forceinline__ float slot_value(const uint32_t (&w)[P], int i) {
     return (float)((int)(v & ((1u << P) - 1u)) - (1 << (P - 1)));
 }
 
-// cos and sin of an angle given in fp64 (token position times frequency, up to ~1e6 rad): reduced to [-pi, pi]
-// in fp64, evaluated in fp32.
-__device__ __forceinline__ void sincos_reduced(double angle, float* sn, float* cs) {
-    const double k = rint(angle * 0.15915494309189535);                        // 1 / (2 pi)
-    const double r = fma(-k, 2.4492935982947064e-16, fma(-k, 6.283185307179586, angle));   // 2 pi in two terms
-    sincosf((float)r, sn, cs);
-}
-
 // ROPE: the cache holds keys as they were before the rotary embedding (Sec. III par. 2); the rotation of
 // token t's key to position t is moved onto the query: q . R_t k = (R_t^T q) . k, and R_t^T q is carried from
 // token to token by a fixed rotation (the lane's tokens are 8 apart).

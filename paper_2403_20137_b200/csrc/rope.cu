@@ -27,28 +27,37 @@ __global__ void __launch_bounds__(kHeadDim) rope_tables(const int32_t* __restric
     sign[h * d + j] = sg;
 }
 
-template <typename T> __device__ __forceinline__ double ld(const T* p);
-template <> __device__ __forceinline__ double ld<float>(const float* p) { return (double)*p; }
-template <> __device__ __forceinline__ double ld<__nv_bfloat16>(const __nv_bfloat16* p) { return (double)__bfloat162float(*p); }
-template <typename T> __device__ __forceinline__ void st(T* p, double v);
-template <> __device__ __forceinline__ void st<float>(float* p, double v) { *p = (float)v; }
-template <> __device__ __forceinline__ void st<__nv_bfloat16>(__nv_bfloat16* p, double v) { *p = __float2bfloat16_rn((float)v); }
+template <typename T> __device__ __forceinline__ float ld(const T* p);
+template <> __device__ __forceinline__ float ld<float>(const float* p) { return *p; }
+template <> __device__ __forceinline__ float ld<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void st(T* p, float v);
+template <> __device__ __forceinline__ void st<float>(float* p, float v) { *p = v; }
+template <> __device__ __forceinline__ void st<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 
-// y[j] = x[j] cos(m theta_j) + sign_j x[partner_j] sin(m theta_j); the angle is formed in fp64 (positions reach
-// tens of thousands of radians, beyond what an fp32 product resolves).  One thread block per (row, head).
+// y[j] = x[j] cos(m theta_j) + sign_j x[partner_j] sin(m theta_j).  The angle is formed and reduced to [-pi, pi]
+// in fp64 (positions reach tens of thousands of radians, beyond what an fp32 product resolves); sine, cosine and
+// the two products are fp32.  A thread keeps one (head, slot) and walks kRopeRows rows, so the tables are read once.
+constexpr int kRopeRows = 32;
 template <typename T>
-__global__ void __launch_bounds__(kHeadDim) rope_apply(const T* __restrict__ x, const int32_t* __restrict__ pos, int n_heads,
-                                                       const double* __restrict__ theta, const int32_t* __restrict__ partner,
-                                                       const float* __restrict__ sign, T* __restrict__ y) {
+__global__ void __launch_bounds__(kHeadDim) rope_apply(const T* __restrict__ x, const int32_t* __restrict__ pos, int64_t n_rows,
+                                                       int n_heads, const double* __restrict__ theta,
+                                                       const int32_t* __restrict__ partner, const float* __restrict__ sign,
+                                                       T* __restrict__ y) {
     constexpr int D = kHeadDim;
-    const int64_t row = blockIdx.x;
     const int h = blockIdx.y, j = threadIdx.x;
-    const T* xr = x + (row * n_heads + h) * D;
-    const double ang = (double)pos[row] * theta[h * D + j];
-    double sn, cs;
-    sincos(ang, &sn, &cs);
-    const double v = ld<T>(xr + j) * cs + (double)sign[h * D + j] * ld<T>(xr + (partner[h * D + j] & (D - 1))) * sn;
-    st<T>(y + (row * n_heads + h) * D + j, v);
+    const double th = theta[h * D + j];
+    const int pj = partner[h * D + j] & (D - 1);
+    const float sg = sign[h * D + j];
+    const int64_t r0 = (int64_t)blockIdx.x * kRopeRows;
+    const int64_t r1 = r0 + kRopeRows < n_rows ? r0 + kRopeRows : n_rows;
+#pragma unroll 4
+    for (int64_t row = r0; row < r1; ++row) {
+        const T* xr = x + (row * n_heads + h) * D;
+        float sn, cs;
+        sincos_reduced((double)pos[row] * th, &sn, &cs);
+        const float v = fmaf(ld<T>(xr + j), cs, sg * ld<T>(xr + pj) * sn);
+        st<T>(y + (row * n_heads + h) * D + j, v);
+    }
 }
 
 }  // namespace
@@ -82,13 +91,13 @@ extern "C" kvbfp_status kvbfp_rope_apply(const void* x, kvbfp_dtype dt, int64_t 
     for (const void* p : ptrs)
         if (!aligned16(p)) return KVBFP_ERR_ALIGNMENT;
     if (n_rows == 0) return KVBFP_OK;
-    dim3 grid((unsigned)n_rows, (unsigned)n_heads);
+    dim3 grid((unsigned)((n_rows + kRopeRows - 1) / kRopeRows), (unsigned)n_heads);
     cudaStream_t s = (cudaStream_t)stream;
     if (dt == KVBFP_F32)
-        rope_apply<float><<<grid, kHeadDim, 0, s>>>((const float*)x, positions, n_heads, theta, partner, sign, (float*)y);
+        rope_apply<float><<<grid, kHeadDim, 0, s>>>((const float*)x, positions, n_rows, n_heads, theta, partner, sign, (float*)y);
     else
-        rope_apply<__nv_bfloat16><<<grid, kHeadDim, 0, s>>>((const __nv_bfloat16*)x, positions, n_heads, theta, partner, sign,
-                                                            (__nv_bfloat16*)y);
+        rope_apply<__nv_bfloat16><<<grid, kHeadDim, 0, s>>>((const __nv_bfloat16*)x, positions, n_rows, n_heads, theta, partner,
+                                                            sign, (__nv_bfloat16*)y);
     KVBFP_LAUNCH_CHECK("rope_apply");
     return KVBFP_OK;
 }
