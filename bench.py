@@ -467,14 +467,16 @@ def main():
         "data": "synthetic",
         "config": {"workload": workload_name(w), "per_gpu_batch": Bn, "decode_kernel": kernel,
                    "l2": f"inputs larger than L2: {alg / 1e6:.0f} MB of cache read per step vs 126 MB L2",
-                   "device_status_flags": flags, "e2e_matches_device_path": e2e_ok},
+                   "device_status_flags": flags, "e2e_matches_device_path": e2e_ok,
+                   "tokens_per_s_if_32_layers": value / 32.0},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": (ms_e2e / args.steps) if n_e2e else None},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic_per_launch(kernel, w),
-                     "algorithmic_bytes": alg, "kernel_ms": kernel_ms, "peak_source": peak_src},
+                     "algorithmic_bytes": alg, "kernel_ms": kernel_ms, "peak_source": peak_src,
+                     "frac_of_nominal_8000_GBs": achieved / 8000.0},
         "extras": extras or None,
     }
     if not args.no_cpu_baseline and world == 1:
