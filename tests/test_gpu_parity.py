@@ -106,6 +106,38 @@ def test_append_bit_exact_format_grid(oracle, dtype, p, n):
     assert np.array_equal(host(B.dequant(gc, "k", 0, 1, 20, 7)).astype(np.float64), ref)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("p", P_GRID)
+@pytest.mark.parametrize("n", N_GRID)
+@pytest.mark.parametrize("heads", [3, 8])
+def test_append_many_tokens_bit_exact(oracle, dtype, p, n, heads):
+    """The cache write on many tokens (several grid strides of the kernel): the adversarial rows tiled to a few
+    thousand tokens over three sequences, two head counts, K permuted, V not, ragged start positions, one sequence
+    that does not fit."""
+    base_k, base_v = adversarial_rows(dtype, seed=4), adversarial_rows(dtype, seed=5)      # [1, 96, 2, 128]
+    reps = 9
+    k = base_k.repeat(3, reps, (heads + 1) // 2, 1)[:, :, :heads].contiguous()               # [3, 864, heads, 128]
+    v = base_v.repeat(3, reps, (heads + 1) // 2, 1)[:, :, :heads].contiguous()
+    k[1] = k[1].flip(0)                                                                      # sequences differ
+    v[2] = v[2].flip(1)
+    T = k.shape[1]
+    rng = np.random.default_rng(6)
+    perm_k = np.stack([rng.permutation(128) for _ in range(heads)]).astype(np.int32)
+    S_max = 1024
+    start = [0, 160, 512]                                                                    # 512 + 864 > 1024: skipped whole
+    gc = B.Cache(3, heads, 128, S_max, n, p, fill=0x5A)
+    B.append(gc, dev(k), dev(v), dev(torch.tensor(start, dtype=torch.int32)), dev(torch.from_numpy(perm_k)))
+    assert B.device_status() == B.FLAG_POSITION
+    assert bool((gc.k_mant[2] == 0x5A).all()) and bool((gc.v_exp[2] == 0x5A).all())
+    oc = oracle.Cache(2, heads, 128, S_max, n, p)
+    oracle.append(oc, W.to_oracle(k[:2]), W.to_oracle(v[:2]), dtype, np.array(start[:2], np.int32), perm_k)
+    for b in range(2):
+        sl = slice(start[b], start[b] + T)
+        for name in ("k_mant", "k_exp", "v_mant", "v_exp"):
+            assert np.array_equal(host(getattr(gc, name)[b, :, sl]), getattr(oc, name)[b, :, sl]), f"{name} differs for batch {b}"
+    assert bool((gc.k_mant[1, :, :160] == 0x5A).all()) and bool((gc.v_mant[0, :, T:] == 0x5A).all())
+
+
 def test_append_identity_and_single_plane(oracle):
     w = W.CONFIGS[2]
     k, v = W.make_kv(w, n_tokens=50)
