@@ -27,6 +27,8 @@
 // the multiply-add pipe was measured slower on B200; the switch is kept, off.)
 #include <math.h>
 
+#include <atomic>
+
 #include "decode.cuh"
 #include "ptx.cuh"
 
@@ -613,12 +615,12 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(Decode
 template <int P, int N, int NT>
 kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s) {
     using G_ = Geo<P, N>;
-    static bool attr_set[64] = {false};
+    static std::atomic<bool> attr_set[64];      // per device; setting the attribute twice is harmless
     int dev = 0;
     KVBFP_CUDA(cudaGetDevice(&dev));
-    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+    if (dev >= 0 && dev < 64 && !attr_set[dev].load(std::memory_order_acquire)) {
         KVBFP_CUDA(cudaFuncSetAttribute(decode_mma<P, N, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_::template smem_bytes<NT>()));
-        attr_set[dev] = true;
+        attr_set[dev].store(true, std::memory_order_release);
     }
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
     make_qfrag<P><<<n_pre, 32, 0, s>>>(a, NT);

@@ -19,6 +19,7 @@
 //   4-bit kernel); 2^(D - 138) is applied in fp32 to the partial result.  Softmax weights are (hi, lo) fp16 pairs.
 #include <math.h>
 
+#include <atomic>
 #include <type_traits>
 
 #include "decode.cuh"
@@ -514,17 +515,18 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
 template <int N, int NT>
 kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     using G_ = Geo8<N>;
-    static int resident[64] = {0};          // thread blocks that fit the whole device, per device
+    static std::atomic<int> resident[64];   // thread blocks that fit the whole device, per device (0 = not asked yet;
+                                            // two host threads asking at once store the same number)
     int dev = 0;
     KVBFP_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return KVBFP_ERR_UNSUPPORTED;
-    if (!resident[dev]) {
+    if (!resident[dev].load(std::memory_order_acquire)) {
         KVBFP_CUDA(cudaFuncSetAttribute(decode_mma8<N, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_::SMEM_BYTES));
         int per_sm = 0, n_sm = 0;
         KVBFP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_mma8<N, NT>, kWarps * 32, G_::SMEM_BYTES));
         KVBFP_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
         if (per_sm < 1 || n_sm < 1) return KVBFP_ERR_CUDA;
-        resident[dev] = per_sm * n_sm;
+        resident[dev].store(per_sm * n_sm, std::memory_order_release);
     }
     int32_t* qmeta = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
                                                (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
@@ -533,7 +535,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     KVBFP_LAUNCH_CHECK("make_qfrag8i");
     DecodeArgs b;
     int grid = 0;
-    const kvbfp_status st = plan_persistent(a, kItemFine, resident[dev], kWarps, &b, split, &grid);
+    const kvbfp_status st = plan_persistent(a, kItemFine, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
     if (st != KVBFP_OK) return st;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);

@@ -7,6 +7,7 @@
 // that workspace in a fixed array that is part of the library image, so the caller passes inputs
 // and outputs only.  The array costs kStaticScratchBytes of device memory on every GPU that loads
 // the library, for as long as the process lives.
+#include <atomic>
 #include "common.cuh"
 
 namespace kvbfp {
@@ -21,17 +22,17 @@ static __device__ __align__(256) uint8_t g_decode_scratch[kStaticScratchBytes];
 // Device address of the array on the current device, looked up once per device.
 kvbfp_status scratch_address(void** out) {
     constexpr int kMaxDev = 64;
-    static void* cache[kMaxDev] = {nullptr};
+    static std::atomic<void*> cache[kMaxDev];      // two host threads asking at once store the same address
     int dev = 0;
     KVBFP_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDev) return KVBFP_ERR_UNSUPPORTED;
-    if (!cache[dev]) {
+    if (!cache[dev].load(std::memory_order_acquire)) {
         void* p = nullptr;
         KVBFP_CUDA(cudaGetSymbolAddress(&p, g_decode_scratch));
         if (!p) return KVBFP_ERR_CUDA;
-        cache[dev] = p;
+        cache[dev].store(p, std::memory_order_release);
     }
-    *out = cache[dev];
+    *out = cache[dev].load(std::memory_order_relaxed);
     return KVBFP_OK;
 }
 

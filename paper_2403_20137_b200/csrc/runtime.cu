@@ -23,16 +23,16 @@ void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_r
 
 kvbfp_status status_word(uint32_t** ptr) {
     constexpr int kMaxDev = 64;
-    static uint32_t* cache[kMaxDev] = {nullptr};
+    static std::atomic<uint32_t*> cache[kMaxDev];      // per device; two threads asking at once store the same address
     int dev = 0;
     KVBFP_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDev) return KVBFP_ERR_UNSUPPORTED;
-    if (!cache[dev]) {
+    if (!cache[dev].load(std::memory_order_acquire)) {
         uint32_t* p = nullptr;
         KVBFP_CUDA(cudaGetSymbolAddress((void**)&p, g_status_word));
-        cache[dev] = p;
+        cache[dev].store(p, std::memory_order_release);
     }
-    *ptr = cache[dev];
+    *ptr = cache[dev].load(std::memory_order_relaxed);
     return KVBFP_OK;
 }
 
