@@ -37,7 +37,7 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.6257, "sources_sha256": "0c678817c0b4588a6132ddd89feeb2846858642a7213e17d2e872026394670cc"}}
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.0515, "sources_sha256": "7909436b9e20135e8d5fd36e634f02d51b99bbbd3bff91496a211fac806cec94"}}
 KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
 
 
