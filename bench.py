@@ -33,12 +33,15 @@ from paper_2403_20137_b200 import workloads as W  # noqa: E402
 METRIC = "decode_attn_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM traffic of the dominant kernel from one ncu capture (profiles/decode_mma4_b4_s8192_ncu_full.md):
+# DRAM traffic of the dominant kernel from one ncu capture (profiles/decode_mma4_b4_s8192_ncu_full.md; the 8-bit
+# kernel: profiles/other_decode_kernels_b4_s8192_ncu_sections.md):
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.0515, "sources_sha256": "7909436b9e20135e8d5fd36e634f02d51b99bbbd3bff91496a211fac806cec94"}}
-KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.0515, "block": 32, "mant_bits": 4, "sources_sha256": "7909436b9e20135e8d5fd36e634f02d51b99bbbd3bff91496a211fac806cec94"},
+           "decode_mma8": {"bytes_per_unit": 264.3372, "block": 32, "mant_bits": 8, "sources_sha256": "0e0ae313fe6df113eeef12d6dc9031be944ef871e159f7e0f2dd54418cc1c5ce"}}
+KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],
+                  "decode_mma8": ["paper_2403_20137_b200/csrc/decode_mma8.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
 
 
 def sources_hash(kernel):
@@ -51,9 +54,10 @@ def sources_hash(kernel):
 
 def traffic_per_launch(kernel, w):
     """DRAM bytes of one launch, scaled from the capture by the units processed; None when there is no capture for
-    this kernel and format (the capture is of block 32, 4-bit mantissas) or the kernel has changed since."""
+    this kernel and format or the kernel has changed since."""
     t = TRAFFIC.get(kernel)
-    if not t or not t["bytes_per_unit"] or (w.block, w.mant_bits) != (32, 4) or t["sources_sha256"] != sources_hash(kernel):
+    if not t or not t["bytes_per_unit"] or (w.block, w.mant_bits) != (t["block"], t["mant_bits"]) or \
+            t["sources_sha256"] != sources_hash(kernel):
         return None
     return t["bytes_per_unit"] * decode_units(w)
 
