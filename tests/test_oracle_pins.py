@@ -39,6 +39,31 @@ def test_powers_of_two_round_trip(oracle, p):
                 assert oracle.bfp_value(M[j], e8, p) == x[j]
 
 
+@pytest.mark.parametrize("p", [4, 6, 8])
+def test_cast_symmetries(oracle, p):
+    """What the cast of Sec. II-B must commute with, whatever its internals: a power-of-two scaling moves the shared
+    exponent and nothing else, a sign flip negates the mantissas (the range is symmetric and ties go to even), and a
+    permutation inside the block permutes the mantissas (the exponent comes from the maximum alone)."""
+    rng = np.random.default_rng(31 + p)
+    for _ in range(200):
+        n = int(rng.choice([16, 32, 64, 128]))
+        x = (rng.standard_normal(n) * 2.0 ** rng.integers(-20, 20)).astype(np.float32).astype(np.float64)
+        x[rng.integers(0, n)] *= 1.0 + rng.integers(0, 30)                    # sometimes an outlier
+        grid = rng.integers(-8, 9, size=n) * 2.0 ** -3                        # plus values that sit on exact ties
+        if rng.random() < 0.3:
+            x = grid
+        e8, M = oracle.bfp_cast_block(x, p)
+        k = int(rng.integers(-40, 40))
+        e8s, Ms = oracle.bfp_cast_block(np.ldexp(x, k), p)
+        if e8 > 0 and 0 < e8 + k < 255:
+            assert e8s == e8 + k and np.array_equal(Ms, M)
+        e8n, Mn = oracle.bfp_cast_block(-x, p)
+        assert e8n == e8 and np.array_equal(Mn, -np.asarray(M))
+        perm = rng.permutation(n)
+        e8p, Mp = oracle.bfp_cast_block(x[perm], p)
+        assert e8p == e8 and np.array_equal(Mp, np.asarray(M)[perm])
+
+
 def test_zero_and_subnormal_blocks(oracle):
     e8, M = oracle.bfp_cast_block(np.zeros(16), 4)
     assert e8 == 0 and not M.any()
