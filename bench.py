@@ -295,6 +295,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the batch size (small cases for profiling)")
     ap.add_argument("--seq", type=int, default=0, help="override the cached sequence length")
+    ap.add_argument("--q-heads", type=int, default=0, help="override the number of query heads (a multiple of the KV heads)")
     ap.add_argument("--mant-bits", type=int, default=0, choices=[0, 4, 6, 8])
     ap.add_argument("--block", type=int, default=0, choices=[0, 16, 32, 64, 128])
     ap.add_argument("--chunk", type=int, default=0, help="tokens per sequence chunk (0 = library default)")
@@ -306,7 +307,7 @@ def main():
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
     over = {k: v for k, v in (("batch", args.batch), ("seq", args.seq), ("mant_bits", args.mant_bits),
-                              ("block", args.block)) if v}
+                              ("block", args.block), ("n_q_heads", args.q_heads)) if v}
     if over:
         w = dataclasses.replace(w, **over)
 
