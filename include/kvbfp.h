@@ -62,7 +62,8 @@ typedef enum { KVBFP_STAT_MAXABS = 0, KVBFP_STAT_L2 = 1 } kvbfp_stat;
 /* Bits of the device status word. */
 enum {
     KVBFP_FLAG_NONFINITE = 1u,     /* an input element was Inf or NaN                        */
-    KVBFP_FLAG_POSITION = 2u,      /* start_pos + n_new or seq_len beyond max_seq: skipped   */
+    KVBFP_FLAG_POSITION = 2u,      /* append: start_pos + n_new beyond max_seq, the sequence's rows are skipped;
+                                      decode: a seq_len beyond max_seq is read as max_seq, a negative one as 0 */
     KVBFP_FLAG_LEN_HINT = 4u,      /* a seq_len exceeded max_len_hint: tokens past it unread */
     KVBFP_FLAG_WAIT_TIMEOUT = 8u   /* an on-chip copy did not complete within its wait bound */
 };
@@ -288,6 +289,27 @@ kvbfp_status kvbfp_decode_step_host(const kvbfp_cache* cache, const void* k_new_
                                     float* out_host, void* staging, size_t staging_bytes,
                                     void* workspace, size_t workspace_bytes, uint32_t flags,
                                     void* stream);
+
+/*
+ * Diagnostics of the work split behind kvbfp_decode_attn (host only: nothing is launched, no device is touched).
+ * The persistent kernels lay the sequence pieces ("items") of all (batch, kv head) pairs out pair-major, cut them
+ * into one contiguous range per resident warp, and let every range write one partial result per pair it touches;
+ * the merge finds those partial results again with the same integer arithmetic.  These calls expose that arithmetic
+ * as the kernels use it, so that it can be checked on its own.
+ *   kvbfp_split_plan         for `pairs` pairs of at most `len_cap` tokens in chunks of `chunk` tokens (a multiple of
+ *                            128), items of `fine_tokens` tokens where the plan allows them, on a device that holds
+ *                            `capacity_blocks` thread blocks of `warps_per_block` warps:
+ *                            out6 = {grid, n_warps, item_tokens, items_per_pair, range_items, range_extra}
+ *   kvbfp_split_range_start  first item of range w (the first range_extra ranges hold range_items + 1 items)
+ *   kvbfp_split_range_of     the range that holds item x
+ *   kvbfp_split_partial_slot the chunk-sized slot (n_chunks per pair) that receives the partial result of a run
+ *                            whose first item within its pair is `item`
+ */
+kvbfp_status kvbfp_split_plan(int32_t pairs, int32_t len_cap, int32_t chunk, int32_t fine_tokens,
+                              int32_t capacity_blocks, int32_t warps_per_block, int32_t* out6);
+int32_t kvbfp_split_range_start(int32_t w, int32_t range_items, int32_t range_extra);
+int32_t kvbfp_split_range_of(int32_t x, int32_t range_items, int32_t range_extra);
+int32_t kvbfp_split_partial_slot(int32_t item, int32_t item_tokens, int32_t chunk, int32_t n_chunks);
 
 /*
  * Profiling aid.  After this call, every kvbfp_decode_attn issued from the calling thread records

@@ -24,7 +24,8 @@ EXPORTS = ["kvbfp_version", "kvbfp_status_string", "kvbfp_last_cuda_error", "kvb
            "kvbfp_decode_workspace_bytes", "kvbfp_decode_attn", "kvbfp_device_status",
            "kvbfp_launch_count", "kvbfp_step_staging_bytes", "kvbfp_decode_step_host",
            "kvbfp_profile_decode_events", "kvbfp_static_scratch_bytes", "kvbfp_decode_attn_static",
-           "kvbfp_rope_tables", "kvbfp_rope_apply", "kvbfp_decode_attn_rope"]
+           "kvbfp_rope_tables", "kvbfp_rope_apply", "kvbfp_decode_attn_rope", "kvbfp_split_plan",
+           "kvbfp_split_range_start", "kvbfp_split_range_of", "kvbfp_split_partial_slot"]
 
 
 class KvbfpError(RuntimeError):
@@ -59,12 +60,13 @@ def lib_path():
 
 
 def lib():
-    """Load (building in-tree if the sources are newer) the CUDA library; raises if impossible."""
+    """Load the CUDA library, first rebuilding it in-tree unless it was built from the sources as they
+    are now (a hash of the sources is kept beside the binary); raises if that is impossible."""
     global _lib
     if _lib is None:
         path = os.environ.get("KVBFP_LIB") or _build.LIB      # KVBFP_LIB: another build of the same library
-        if path == _build.LIB and (not os.path.exists(path) or os.environ.get("KVBFP_REBUILD")):
-            path = _build.build()
+        if path == _build.LIB:
+            path = _build.build()                             # returns at once when the binary is current
         L = C.CDLL(path)
         L.kvbfp_version.restype = C.c_int32
         L.kvbfp_status_string.restype = C.c_char_p
@@ -104,6 +106,12 @@ def lib():
                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.kvbfp_rope_apply.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        L.kvbfp_split_plan.argtypes = [C.c_int32] * 6 + [C.POINTER(C.c_int32)]
+        for name in ("kvbfp_split_range_start", "kvbfp_split_range_of"):
+            getattr(L, name).argtypes = [C.c_int32] * 3
+            getattr(L, name).restype = C.c_int32
+        L.kvbfp_split_partial_slot.argtypes = [C.c_int32] * 4
+        L.kvbfp_split_partial_slot.restype = C.c_int32
         _lib = L
     return _lib
 

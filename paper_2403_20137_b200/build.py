@@ -1,4 +1,5 @@
 """Compile the CUDA library in-tree: ``csrc/*.cu`` -> ``libkvbfp.so`` (sm_100a only)."""
+import hashlib
 import os
 import subprocess
 import sys
@@ -18,9 +19,28 @@ def sources():
     return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
 
 
-def _deps_mtime():
-    files = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "kvbfp.h"), __file__]
-    return max(os.path.getmtime(f) for f in files)
+STAMP = LIB + ".sources"     # hash of the sources the library was built from (kept beside it, travels with it)
+
+
+def sources_hash() -> str:
+    """Hash over everything the library is compiled from; file times do not enter (a copy of the tree may reset them)."""
+    files = sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh")))
+    files += [os.path.join(INCLUDE, "kvbfp.h"), os.path.abspath(__file__)]
+    h = hashlib.sha256()
+    for f in files:
+        h.update(os.path.basename(f).encode() + b"\0")
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
+
+
+def is_current() -> bool:
+    """True when libkvbfp.so exists and was built from the sources as they are now."""
+    try:
+        with open(STAMP) as fh:
+            return os.path.exists(LIB) and fh.read().strip() == sources_hash()
+    except OSError:
+        return False
 
 
 def _compile(src, obj_dir=None, extra=()):
@@ -36,8 +56,9 @@ def _compile(src, obj_dir=None, extra=()):
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _deps_mtime():
+    if not force and is_current():
         return LIB
+    stamp = sources_hash()
     os.makedirs(OBJ_DIR, exist_ok=True)
     if force:
         for f in os.listdir(OBJ_DIR):
@@ -52,19 +73,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
                         "-lcudart"], capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
+    with open(STAMP, "w") as fh:
+        fh.write(stamp + "\n")
     return LIB
-
-
-def build_variant(out, defines, obj_dir):
-    """Development aid: the same sources with extra -D flags into another .so (tuning sweeps)."""
-    os.makedirs(obj_dir, exist_ok=True)
-    extra = tuple("-D" + d for d in defines)
-    with ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as ex:
-        results = list(ex.map(lambda src: _compile(src, obj_dir, extra), sources()))
-    objs = [o for o, _ in results]
-    subprocess.run(["nvcc", "-shared", "-o", out, *objs, "-gencode", "arch=compute_100a,code=sm_100a", "-lcudart"],
-                   check=True)
-    return out
 
 
 if __name__ == "__main__":

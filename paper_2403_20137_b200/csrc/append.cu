@@ -151,9 +151,12 @@ template <int P, int N, typename T>
 kvbfp_status launch(const AppendArgs& a, int64_t n_rows, cudaStream_t s) {
     const int64_t n_tok = (int64_t)a.batch * a.n_new;
     const int64_t want = (n_tok + kTokPerCta - 1) / kTokPerCta;
-    const int gx = (int)(want < 148 * 16 ? want : 148 * 16);
+    int n_sm = 0;
+    const kvbfp_status st = sm_count(&n_sm);
+    if (st != KVBFP_OK) return st;
+    const int gx = (int)(want < n_sm * 16 ? want : n_sm * 16);
     (void)n_rows;
-    int hs = (int)((148 * 4 + gx - 1) / gx);              // enough thread blocks to fill the machine
+    int hs = (int)((n_sm * 4 + gx - 1) / gx);             // enough thread blocks to fill the machine
     if (hs > a.n_heads) hs = a.n_heads;
     if (hs < 1) hs = 1;
     dim3 grid(gx, 2, hs);

@@ -159,7 +159,10 @@ kvbfp_status run_calibrate(const void* x, int64_t n_tokens, int n_heads, kvbfp_s
         unit = vec_per_row / a;
     }
     int64_t want = (n_vec + kThreads - 1) / kThreads;
-    int64_t cap = 148 * 8;
+    int n_sm = 0;
+    const kvbfp_status sm_st = sm_count(&n_sm);
+    if (sm_st != KVBFP_OK) return sm_st;
+    int64_t cap = (int64_t)n_sm * 8;
     int64_t g = want < cap ? want : cap;
     g = ((g + unit - 1) / unit) * unit;
     if (g < unit) g = unit;

@@ -18,6 +18,8 @@ kvbfp_status cuda_fail(cudaError_t e, const char* what);
 // Address of the device status word of the current device (no allocation: a __device__ symbol).
 kvbfp_status status_word(uint32_t** ptr);
 void count_launch(int n = 1);
+// Number of SMs of the current device (asked once per device); grids are sized in multiples of it.
+kvbfp_status sm_count(int* n);
 
 #define KVBFP_CUDA(call)                                                         \
     do {                                                                         \

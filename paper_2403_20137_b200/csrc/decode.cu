@@ -130,6 +130,7 @@ kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype 
     if (n_q_heads < 1 || n_q_heads % f.n_kv_heads != 0) return KVBFP_ERR_INVALID_ARG;
     const int group = n_q_heads / f.n_kv_heads;
     if (group > 8) return KVBFP_ERR_UNSUPPORTED;
+    if ((int64_t)f.batch * n_q_heads > (1 << 28)) return KVBFP_ERR_UNSUPPORTED;     // row counts are 32-bit in the kernels
     if (q_dt != KVBFP_F32 && q_dt != KVBFP_BF16) return KVBFP_ERR_INVALID_ARG;
     if (q_mant_bits != 0 && q_mant_bits != 8) return KVBFP_ERR_UNSUPPORTED;
     if (max_len_hint < 0 || !(softmax_scale >= 0.f) || isinf(softmax_scale)) return KVBFP_ERR_INVALID_ARG;
@@ -174,7 +175,10 @@ kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype 
         chunk = kMinChunk;      // the persistent kernel balances by item count: finest items, one partial per range
     } else {
         const int64_t pairs = (int64_t)f.batch * f.n_kv_heads;
-        const int64_t target_items = 148 * 16 * 4;
+        int n_sm = 0;
+        st = sm_count(&n_sm);
+        if (st != KVBFP_OK) return st;
+        const int64_t target_items = (int64_t)n_sm * 16 * 4;
         int64_t want = (target_items + pairs - 1) / pairs;
         if (want < 1) want = 1;
         int64_t per = (a.len_cap + want - 1) / want;
@@ -185,7 +189,6 @@ kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype 
     a.n_chunks = (a.len_cap + chunk - 1) / chunk;
     st = status_word(&a.status);
     if (st != KVBFP_OK) return st;
-    a.mulhi4 = 1u << 28; a.mulhi8 = 1u << 24; a.mulhi12 = 1u << 20;
 
     cudaStream_t s = (cudaStream_t)stream;
     a.item_tokens = a.chunk;
@@ -226,6 +229,38 @@ extern "C" kvbfp_status kvbfp_decode_attn_rope(const kvbfp_cache* cache, const v
     if (!theta || !partner || !sign) return KVBFP_ERR_INVALID_ARG;
     return kvbfp::decode_common(cache, q, q_dt, n_q_heads, seq_lens, max_len_hint, perm_k, inv_perm_v, softmax_scale, 0,
                                 theta, partner, sign, out, workspace, workspace_bytes, flags, stream);
+}
+
+// ---- diagnostics: the split arithmetic itself, callable from the host ----------------------------------------
+extern "C" kvbfp_status kvbfp_split_plan(int32_t pairs, int32_t len_cap, int32_t chunk, int32_t fine_tokens,
+                                         int32_t capacity_blocks, int32_t warps_per_block, int32_t* out6) {
+    using namespace kvbfp;
+    if (!out6 || pairs < 1 || len_cap < 1 || chunk < kMinChunk || chunk % kMinChunk != 0 || fine_tokens < 1 ||
+        capacity_blocks < 1 || warps_per_block < 1)
+        return KVBFP_ERR_INVALID_ARG;
+    DecodeArgs a{};
+    a.fmt.batch = pairs;
+    a.fmt.n_kv_heads = 1;
+    a.len_cap = len_cap;
+    a.chunk = chunk;
+    a.n_chunks = (len_cap + chunk - 1) / chunk;
+    DecodeArgs b;
+    Split split;
+    int grid = 0;
+    const kvbfp_status st = plan_persistent(a, fine_tokens, capacity_blocks, warps_per_block, &b, &split, &grid);
+    if (st != KVBFP_OK) return st;
+    out6[0] = grid; out6[1] = split.n_warps; out6[2] = split.item_tokens; out6[3] = split.items_per_pair;
+    out6[4] = split.range_items; out6[5] = split.range_extra;
+    return KVBFP_OK;
+}
+extern "C" int32_t kvbfp_split_range_start(int32_t w, int32_t range_items, int32_t range_extra) {
+    return kvbfp::range_start(w, range_items, range_extra);
+}
+extern "C" int32_t kvbfp_split_range_of(int32_t x, int32_t range_items, int32_t range_extra) {
+    return kvbfp::range_of(x, range_items, range_extra);
+}
+extern "C" int32_t kvbfp_split_partial_slot(int32_t item, int32_t item_tokens, int32_t chunk, int32_t n_chunks) {
+    return kvbfp::partial_slot(item, item_tokens, chunk, n_chunks);
 }
 
 extern "C" kvbfp_status kvbfp_profile_decode_events(void* start_event, void* stop_event) {

@@ -35,9 +35,6 @@ struct DecodeArgs {
     const int32_t* rope_partner;
     const float* rope_sign;
     uint32_t* status;
-    // 2^(32-k): multiplying by these and keeping the high word is a right shift by k that runs on the
-    // multiply-add pipe instead of the integer pipe (passed at run time so that it stays a multiply)
-    uint32_t mulhi4, mulhi8, mulhi12;
 };
 
 kvbfp_status launch_decode_simt(const DecodeArgs& a, cudaStream_t s);
@@ -64,23 +61,25 @@ __host__ __device__ __forceinline__ int range_of(int x, int range_items, int ran
 // Slot (chunk-sized, n_chunks per pair) that receives the partial of a run whose first item within its pair
 // is `item`.  Items are whole chunks, or half chunks: then two runs can start in the first chunk of a pair (one
 // that holds only item 0, the next from item 1 on), so odd items round up; ranges hold four items or more, so
-// no other two runs start within two items of each other and the clamp at the last slot is safe as well.
+// no other two runs start within two items of each other and the clamp at the last slot is safe as well --
+// provided a pair has two slots or more: with a single chunk per pair, items 0 and 1 would share slot 0, so
+// plan_persistent() never cuts such pairs into half chunks.
 __host__ __device__ __forceinline__ int partial_slot(int item, int item_tokens, int chunk, int n_chunks) {
     if (item_tokens == chunk) return item;
     const int s = (item + 1) >> 1;
     return s < n_chunks ? s : n_chunks - 1;
 }
 // Work split of a persistent kernel (host side).  Items are pieces of `fine_tokens` tokens (half a chunk) when the
-// library chose the chunking (chunk == kMinChunk == 2 * fine_tokens) and every warp still gets five or more of them
-// on average, so four at the least (the ranges then differ by one piece of work at most and partial_slot() keeps
-// the runs' partial results apart); whole chunks otherwise.  The items are cut into one contiguous range per warp
+// library chose the chunking (chunk == kMinChunk == 2 * fine_tokens), a pair has two chunks or more, and every warp
+// still gets five or more items on average, so four at the least (the ranges then differ by one piece of work at
+// most and partial_slot() keeps the runs' partial results apart); whole chunks otherwise.  The items are cut into one contiguous range per warp
 // of min(capacity, blocks needed) thread blocks.  Fills the range fields of `b` and `split`, returns the grid.
 inline kvbfp_status plan_persistent(const DecodeArgs& a, int fine_tokens, int capacity_blocks, int warps_per_block,
                                     DecodeArgs* b, Split* split, int* grid) {
     *b = a;
     const int64_t pairs = (int64_t)a.fmt.batch * a.fmt.n_kv_heads;
     const int fine_per_pair = (a.len_cap + fine_tokens - 1) / fine_tokens;
-    const bool fine = a.chunk == 2 * fine_tokens && a.chunk == kMinChunk &&
+    const bool fine = a.chunk == 2 * fine_tokens && a.chunk == kMinChunk && a.n_chunks >= 2 &&
                       pairs * fine_per_pair >= 5LL * capacity_blocks * warps_per_block;
     b->item_tokens = fine ? fine_tokens : a.chunk;
     b->items_per_pair = fine ? fine_per_pair : a.n_chunks;

@@ -23,8 +23,7 @@
 //
 // The integer pipe (logic ops, shifts, byte permutes) is what limits this kernel: every field is
 // extracted with one three-input logic instruction and block weights come from a 256-entry table in
-// shared memory instead of being rebuilt from the exponent byte.  (Issuing shifts as multiply-high on
-// the multiply-add pipe was measured slower on B200; the switch is kept, off.)
+// shared memory instead of being rebuilt from the exponent byte.
 #include <math.h>
 
 #include <atomic>
@@ -35,31 +34,10 @@
 namespace kvbfp {
 namespace {
 
-// Tuning knobs (compile-time; the defaults are the measured best on B200).
-#ifndef KVBFP_WARPS
-#define KVBFP_WARPS 4
-#endif
-#ifndef KVBFP_MT
-#define KVBFP_MT 2
-#endif
-#ifndef KVBFP_STAGES
-#define KVBFP_STAGES 3
-#endif
-#ifndef KVBFP_SHIFT_MULHI
-#define KVBFP_SHIFT_MULHI 0            // 1: shifts by 4 and 12 as multiply-high on the multiply-add pipe (slower on B200)
-#endif
-#ifndef KVBFP_MIN_CTAS
-#define KVBFP_MIN_CTAS 1               // resident thread blocks per SM the register allocation must allow
-#endif
-#ifndef KVBFP_QF_SMEM
-#define KVBFP_QF_SMEM 0                // 1: keep the query fragments in shared memory instead of registers
-#endif
-#ifndef KVBFP_K_ACC_SPLIT
-#define KVBFP_K_ACC_SPLIT 1            // 1: two independent accumulator chains for the score MMAs
-#endif
-
-constexpr int kWarps = KVBFP_WARPS;
-constexpr int kMT = KVBFP_MT;          // 16-token MMA row tiles per stage
+constexpr int kWarps = 4;
+constexpr int kMT = 2;             // 16-token MMA row tiles per stage
+constexpr int kStages = 3;         // shared-memory stages per warp
+constexpr int kMinCtas = 1;        // resident thread blocks per SM the register allocation must allow
 constexpr int kTile = 16 * kMT;        // tokens per stage
 
 // bf16 bit pattern of 2^(e8 - 127 - (P-2)); subnormal results down to 2^-133 are exact.
@@ -104,22 +82,6 @@ __device__ __forceinline__ uint32_t cvt_pair(uint32_t x, const Wgt& w) {
     return fma_bf16x2(lop3<0xEA>(x, Fmt<P>::mask, Fmt<P>::magic), w.s, w.c);   // (x & mask) | 128.0 in one op
 }
 
-// Right shifts of a packed word by 4, 8 and 12; two of the three run on the multiply-add pipe.
-struct Shifts {
-    uint32_t m4, m12;
-    __device__ __forceinline__ void apply(uint32_t x, uint32_t& x4, uint32_t& x8, uint32_t& x12) const {
-#if KVBFP_SHIFT_MULHI
-        x4 = __umulhi(x, m4);
-        x8 = x >> 8;
-        x12 = __umulhi(x, m12);
-#else
-        x4 = x >> 4;
-        x8 = x >> 8;
-        x12 = x >> 12;
-#endif
-    }
-};
-
 // Slot (within the 128-slot row) that the K-side unpack puts at k-position kk of k-step ks for lane
 // column t; kk = 0..3 stands for k = 2t, 2t+1, 2t+8, 2t+9 of the m16n8k16 fragment.
 template <int P>
@@ -132,11 +94,11 @@ __host__ __device__ __forceinline__ int k_slot(int ks, int t, int kk) {
 // Two A registers (k = 2t..2t+1 and k = 2t+8..2t+9) of k-steps ks and ks+1 (ks even) from a lane's
 // 32-slot chunk w[P].
 template <int P>
-__device__ __forceinline__ void k_pairs2(const uint32_t (&w)[P], int ks, const Wgt& wg, const Shifts& sh,
+__device__ __forceinline__ void k_pairs2(const uint32_t (&w)[P], int ks, const Wgt& wg,
                                          uint32_t (&r)[4]) {
     if (P == 4) {
         uint32_t x4, x8, x12;
-        sh.apply(w[ks >> 1], x4, x8, x12);
+        x4 = w[ks >> 1] >> 4; x8 = w[ks >> 1] >> 8; x12 = w[ks >> 1] >> 12;
         r[0] = cvt_pair<4>(w[ks >> 1], wg);
         r[1] = cvt_pair<4>(x4, wg);
         r[2] = cvt_pair<4>(x8, wg);
@@ -161,13 +123,13 @@ __device__ __forceinline__ void k_pairs2(const uint32_t (&w)[P], int ks, const W
 // V side: registers for MMA row pairs r and r+1 (r even): (slot 2r, 2r+1, 2r+2, 2r+3) x (token pair),
 // from the two tokens' 16-slot pieces wa, wb (P/2 words each).
 template <int P>
-__device__ __forceinline__ void v_pairs2(const uint32_t* wa, const uint32_t* wb, int r, const Wgt& wg, const Shifts& sh,
+__device__ __forceinline__ void v_pairs2(const uint32_t* wa, const uint32_t* wb, int r, const Wgt& wg,
                                          uint32_t (&o)[4]) {
     if (P == 4) {
         // word i = slots 8i..8i+7; halfword h of word i = slots 8i+4h..8i+4h+3 = rows 2r..2r+3 with r = 4i+2h
         const uint32_t x = prmt(wa[r >> 2], wb[r >> 2], ((r >> 1) & 1) ? 0x7632u : 0x5410u);
         uint32_t x4, x8, x12;
-        sh.apply(x, x4, x8, x12);
+        x4 = x >> 4; x8 = x >> 8; x12 = x >> 12;
         o[0] = cvt_pair<4>(x, wg);
         o[1] = cvt_pair<4>(x4, wg);
         o[2] = cvt_pair<4>(x8, wg);
@@ -259,7 +221,7 @@ template <int P, int N>
 struct Geo {
     static constexpr int D = kHeadDim;
     static constexpr int ROW_M = D * P / 8, ROW_E = D / N;
-    static constexpr int STAGES = KVBFP_STAGES;
+    static constexpr int STAGES = kStages;
     static constexpr int KM_OFF = 0;
     static constexpr int VM_OFF = kTile * ROW_M;
     static constexpr int KE_OFF = 2 * kTile * ROW_M;
@@ -268,13 +230,11 @@ struct Geo {
     static constexpr int WARP_BYTES = STAGES * STAGE_BYTES;
     static constexpr int LUT_OFF = kWarps * WARP_BYTES;                 // uint2[256]
     static constexpr int BAR_OFF = LUT_OFF + 256 * 8;
-    static constexpr int QF_OFF = BAR_OFF + kWarps * STAGES * 8;        // uint2[NT][8][32] per warp (optional)
-    static constexpr int QF_WARP_BYTES = 8 * 32 * 8;                    // per n-tile
-    template <int NT> static constexpr int smem_bytes() { return QF_OFF + (KVBFP_QF_SMEM ? kWarps * NT * QF_WARP_BYTES : 0); }
+    template <int NT> static constexpr int smem_bytes() { return BAR_OFF + kWarps * STAGES * 8; }
 };
 
 template <int P, int N, int NT>
-__global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(DecodeArgs a) {
+__global__ void __launch_bounds__(kWarps * 32, kMinCtas) decode_mma(DecodeArgs a) {
     using G_ = Geo<P, N>;
     constexpr int D = kHeadDim, ROW_M = G_::ROW_M, ROW_E = G_::ROW_E, STAGES = G_::STAGES;
     constexpr int NBK = (N == 16) ? 2 : 1;            // blocks inside a K lane chunk of 32 slots
@@ -344,23 +304,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(Decode
         for (int s = 0; s < STAGES && s < n_tiles; ++s) issue(s, s);
     }
 
-    // B fragments of pi(q): 16 registers per n-tile, or a per-warp copy in shared memory
-#if KVBFP_QF_SMEM
-    uint2* qsm = reinterpret_cast<uint2*>(smem + G_::QF_OFF + warp * NT * G_::QF_WARP_BYTES) + lane;
-    {
-        const uint4* src = reinterpret_cast<const uint4*>(a.qfrag) + (((int64_t)b * Hkv + hk) * NT) * (4 * 32);
-#pragma unroll
-        for (int nt = 0; nt < NT; ++nt)
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint4 v = __ldg(src + (nt * 4 + j) * 32 + lane);
-                qsm[(nt * 8 + 2 * j) * 32] = make_uint2(v.x, v.y);
-                qsm[(nt * 8 + 2 * j + 1) * 32] = make_uint2(v.z, v.w);
-            }
-    }
-    __syncwarp();
-#define QF(nt, ks) (qsm[((nt) * 8 + (ks)) * 32])
-#else
+    // B fragments of pi(q): 16 registers per n-tile
     uint2 qf[NT][8];
     {
         const uint4* src = reinterpret_cast<const uint4*>(a.qfrag) + (((int64_t)b * Hkv + hk) * NT) * (4 * 32);
@@ -374,8 +318,6 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(Decode
             }
     }
 #define QF(nt, ks) (qf[nt][ks])
-#endif
-    const Shifts sh{a.mulhi4, a.mulhi12};
 
     float o[NT][8][4];
 #pragma unroll
@@ -441,7 +383,7 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(Decode
                 ga[k] = make_wgt<P>(la.x, la.y);
                 gb[k] = make_wgt<P>(lb.x, lb.y);
             }
-            constexpr int NACC = KVBFP_K_ACC_SPLIT ? 2 : 1;
+            constexpr int NACC = 2;     // two independent accumulator chains for the score MMAs
             float acc[NT][NACC][4];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
@@ -451,8 +393,8 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(Decode
             for (int ks = 0; ks < 8; ks += 2) {
                 const int kb = (NBK == 2) ? (ks >> 2) : 0;
                 uint32_t ra[4], rb[4];
-                k_pairs2<P>(wa, ks, ga[kb], sh, ra);
-                k_pairs2<P>(wb, ks, gb[kb], sh, rb);
+                k_pairs2<P>(wa, ks, ga[kb], ra);
+                k_pairs2<P>(wb, ks, gb[kb], rb);
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     const uint2 q0 = QF(nt, ks), q1 = QF(nt, ks + 1);
@@ -564,8 +506,8 @@ __global__ void __launch_bounds__(kWarps * 32, KVBFP_MIN_CTAS) decode_mma(Decode
 #pragma unroll
             for (int r = 0; r < 8; r += 2) {
                 uint32_t xa[4], xb[4];
-                v_pairs2<P>(vw[0], vw[1], r, gA, sh, xa);
-                v_pairs2<P>(vw[2], vw[3], r, gB, sh, xb);
+                v_pairs2<P>(vw[0], vw[1], r, gA, xa);
+                v_pairs2<P>(vw[2], vw[3], r, gB, xb);
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
                     mma_bf16(o[nt][r], xa[0], xa[1], xb[0], xb[1], pb[nt][0], pb[nt][1]);
@@ -626,6 +568,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s) {
     make_qfrag<P><<<n_pre, 32, 0, s>>>(a, NT);
     KVBFP_LAUNCH_CHECK("make_qfrag");
     const int64_t n_items = (int64_t)a.fmt.batch * a.fmt.n_kv_heads * a.n_chunks;
+    if ((n_items + kWarps - 1) / kWarps > 0x7fffffffLL) return KVBFP_ERR_UNSUPPORTED;     // more thread blocks than a grid holds
     const int grid = (int)((n_items + kWarps - 1) / kWarps);
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);

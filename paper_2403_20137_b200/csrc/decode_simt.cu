@@ -244,6 +244,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_simt(DecodeArgs a) {
 template <int P, int N, bool ROPE>
 kvbfp_status launch(const DecodeArgs& a, cudaStream_t s) {
     const int64_t n_items = (int64_t)a.fmt.batch * a.n_q_heads * a.n_chunks;
+    if ((n_items + kWarps - 1) / kWarps > 0x7fffffffLL) return KVBFP_ERR_UNSUPPORTED;     // more thread blocks than a grid holds
     const int grid = (int)((n_items + kWarps - 1) / kWarps);
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);

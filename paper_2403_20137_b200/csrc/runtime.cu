@@ -21,6 +21,22 @@ kvbfp_status cuda_fail(cudaError_t e, const char* what) {
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
 
+kvbfp_status sm_count(int* n) {
+    constexpr int kMaxDev = 64;
+    static std::atomic<int> cache[kMaxDev];            // per device; 0 = not asked yet
+    int dev = 0;
+    KVBFP_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDev) return KVBFP_ERR_UNSUPPORTED;
+    int v = cache[dev].load(std::memory_order_acquire);
+    if (!v) {
+        KVBFP_CUDA(cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev));
+        if (v < 1) return KVBFP_ERR_CUDA;
+        cache[dev].store(v, std::memory_order_release);
+    }
+    *n = v;
+    return KVBFP_OK;
+}
+
 kvbfp_status status_word(uint32_t** ptr) {
     constexpr int kMaxDev = 64;
     static std::atomic<uint32_t*> cache[kMaxDev];      // per device; two threads asking at once store the same address

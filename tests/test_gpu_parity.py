@@ -111,9 +111,9 @@ def test_append_bit_exact_format_grid(oracle, dtype, p, n):
 @pytest.mark.parametrize("n", N_GRID)
 @pytest.mark.parametrize("heads", [3, 8])
 def test_append_many_tokens_bit_exact(oracle, dtype, p, n, heads):
-    """The cache write on many tokens (several grid strides of the kernel): the adversarial rows tiled to a few
-    thousand tokens over three sequences, two head counts, K permuted, V not, ragged start positions, one sequence
-    that does not fit."""
+    """The cache write on many tokens (many thread blocks, each walking the heads; the token stride of the grid is
+    taken by test_append_config5_sampled): the adversarial rows tiled to a few thousand tokens over three sequences,
+    two head counts, K permuted, V not, ragged start positions, one sequence that does not fit."""
     base_k, base_v = adversarial_rows(dtype, seed=4), adversarial_rows(dtype, seed=5)      # [1, 96, 2, 128]
     reps = 9
     k = base_k.repeat(3, reps, (heads + 1) // 2, 1)[:, :, :heads].contiguous()               # [3, 864, heads, 128]
@@ -230,6 +230,61 @@ def test_calibrate_l2_and_fold(oracle):
     a = wq[:d].astype(np.float64).T @ wk[:d].astype(np.float64)
     b = fq[:d].T @ fk[:d]
     assert np.allclose(a, b, rtol=1e-12, atol=1e-12)
+
+
+@pytest.mark.parametrize("dtype,T,H", [("bf16", 8192, 32), ("f32", 8192, 32), ("bf16", 1 << 20, 8)])
+def test_calibrate_long_inputs_match_oracle(oracle, dtype, T, H):
+    """Token counts at which every thread of the reduction walks its unrolled main loop several times (a thread
+    block covers a few hundred rows per grid stride): config 3's head count in both input types, and config 5's
+    2^20 calibration tokens.  Statistic, permutation and inverse are bit-exact."""
+    import dataclasses
+    w = dataclasses.replace(W.CONFIGS[5 if H == 8 else 3], dtype=dtype)
+    x = W.make_calibration(w, n_tokens=T, device="cuda")
+    st, perm, inv = B.calibrate(x, H, 128)
+    assert B.device_status() == 0
+    st_o, perm_o, inv_o = oracle.calibrate(W.to_oracle(x), dtype, H, 128)
+    assert np.array_equal(host(st).astype(np.float64), st_o)
+    assert np.array_equal(host(perm), perm_o) and np.array_equal(host(inv), inv_o)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_calibrate_l2_long_input(oracle, dtype):
+    """Euclidean-norm statistic over 8192 rows (several grid strides of the fp64 sum kernel)."""
+    rng = np.random.default_rng(15)
+    H, d, rows = 8, 128, 8192
+    x = torch.from_numpy(rng.standard_normal((rows, H, d)).astype(np.float32)).to(W.torch_dtype(dtype))
+    x[:, 3, 17] *= 9.0
+    st, perm, inv = B.calibrate(dev(x), H, d, stat=B.STAT_L2)
+    st_o, perm_o, inv_o = oracle.calibrate(W.to_oracle(x), dtype, H, d, stat=oracle.STAT_L2)
+    assert np.allclose(host(st), st_o, rtol=1e-6, atol=0)
+    gp = host(perm)
+    for h in range(H):      # identical, or differing only between channels whose norms agree to 1e-12
+        for j in np.nonzero(gp[h] != perm_o[h])[0]:
+            assert abs(st_o[h, gp[h, j]] - st_o[h, perm_o[h, j]]) <= 1e-12 * st_o[h, perm_o[h, j]]
+    assert np.array_equal(np.argsort(gp, axis=1), host(inv))
+
+
+@pytest.mark.parametrize("dtype,p,n", [("bf16", 4, 32), ("f32", 8, 16), ("bf16", 6, 64)])
+def test_append_config5_sampled(oracle, dtype, p, n):
+    """The prefill of config 5: 65536 new tokens x 8 KV heads in one call (more tokens than one pass of the grid
+    takes, so thread blocks stride over the tokens), K permuted.  Two sampled heads are compared with the oracle
+    bit for bit over all 65536 rows, K and V planes."""
+    import dataclasses
+    w = dataclasses.replace(W.CONFIGS[5], dtype=dtype)
+    T, H, d = w.seq, w.n_kv_heads, 128
+    dv = torch.device("cuda")
+    k, v = W.make_kv(w, n_tokens=T, device=dv, batch=1)
+    _, perm, _ = B.calibrate(k.reshape(-1, H, d), H, d)
+    cache = B.Cache(1, H, d, T, n, p, device=dv)
+    B.append(cache, k, v, torch.zeros(1, dtype=torch.int32, device=dv), perm_k=perm)
+    assert B.device_status() == 0
+    perm_h = host(perm)
+    for h in (1, H - 1):
+        oc = oracle.Cache(1, 1, d, T, n, p)
+        oracle.append(oc, W.to_oracle(k[:, :, h:h + 1]), W.to_oracle(v[:, :, h:h + 1]), dtype, np.zeros(1, np.int32),
+                      perm_k=perm_h[h:h + 1])
+        for name in ("k_mant", "k_exp", "v_mant", "v_exp"):
+            assert np.array_equal(host(getattr(cache, name)[0, h]), getattr(oc, name)[0, 0]), f"{name} differs, head {h}"
 
 
 # ------------------------------------------------------------------------------- decode attention
@@ -410,8 +465,14 @@ def test_decode_len_hint_flag(oracle):
     b = B.decode_attn(gc, q, dev(torch.tensor([128], dtype=torch.int32)))
     assert B.device_status() == 0
     assert torch.equal(a, b)                               # tokens past the hint were not read
-    B.decode_attn(gc, q, dev(torch.tensor([300], dtype=torch.int32)))
+    # a length beyond the capacity is read as the capacity, a negative one as an empty sequence; both are flagged
+    full = B.decode_attn(gc, q, lens)
+    over = B.decode_attn(gc, q, dev(torch.tensor([300], dtype=torch.int32)))
     assert B.device_status() & B.FLAG_POSITION
+    assert torch.equal(over, full)
+    neg = B.decode_attn(gc, q, dev(torch.tensor([-5], dtype=torch.int32)))
+    assert B.device_status() & B.FLAG_POSITION
+    assert not bool(neg.any())
 
 
 def test_ksort_improves_gpu_cache_quality(oracle):
@@ -499,15 +560,19 @@ def test_decode_over_pre_rotation_keys(oracle, half_split, p, n):
                            impl=B.DECODE_MMA)
 
 
-def _full_size_case(oracle, cfg, sample_pairs):
+def _full_size_case(oracle, cfg, sample_pairs, **over):
     """The benchmark's own launch (full batch, full sequence, library-chosen chunking) with inputs drawn on
-    the GPU; the oracle recomputes sampled (batch, kv head) units one by one from the same raw inputs."""
-    w = W.CONFIGS[cfg]
+    the GPU; the oracle recomputes the permutation from the same calibration tokens and sampled (batch, kv head)
+    units one by one from the same raw inputs."""
+    import dataclasses
+    w = dataclasses.replace(W.CONFIGS[cfg], **over)
     S, Bn, Hkv, Hq, d = w.seq, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim
     G = Hq // Hkv
     dv = torch.device("cuda")
     calib = W.make_calibration(w, device=dv)
     _, perm, _ = B.calibrate(calib, Hkv, d)
+    _, perm_o, _ = oracle.calibrate(W.to_oracle(calib), w.dtype, Hkv, d)
+    assert np.array_equal(host(perm), perm_o), "permutation differs from the oracle's"
     del calib
     k, v = W.make_kv(w, n_tokens=S, device=dv)
     q = W.make_q(w, device=dv)
@@ -519,7 +584,7 @@ def _full_size_case(oracle, cfg, sample_pairs):
     lens = torch.full((Bn,), S, dtype=torch.int32, device=dv)
     out = B.decode_attn(cache, q, lens, perm_k=perm, max_len_hint=S)
     assert B.device_status() == 0
-    perm_h = host(perm)
+    perm_h = perm_o
     worst = 0.0
     for (b, h) in sample_pairs:
         kk = W.to_oracle(k[b:b + 1, :, h:h + 1])
@@ -545,6 +610,26 @@ def test_full_size_config3_sampled(oracle):
 def test_full_size_config4_gqa_sampled(oracle):
     """B8, 32 query heads on 8 KV heads, S32768: two sampled (batch, kv head) units, four query heads each."""
     _full_size_case(oracle, 4, [(0, 0), (7, 5)])
+
+
+def test_full_size_config2_sampled(oracle):
+    """B1, H32, S4096 (a launch that does not fill the machine): three sampled heads."""
+    _full_size_case(oracle, 2, [(0, 0), (0, 13), (0, 31)])
+
+
+@pytest.mark.parametrize("p", [6, 8])
+def test_full_size_config3_mantissa_sweep_sampled(oracle, p):
+    """Config 3's mantissa sweep at full size: the 6-bit and the 8-bit kernels on B16, H32, S8192."""
+    _full_size_case(oracle, 3, [(0, 1), (15, 30), (8, 16)], mant_bits=p)
+
+
+@pytest.mark.parametrize("p", [4, 8])
+def test_group_of_8_long_sequences_sampled(oracle, p):
+    """Eight query heads per KV head (two 8-column tiles per warp), 64 sequences of 4096 tokens on 4 KV heads:
+    256 pairs of 64 items each against about a dozen items per warp, so that many warps' ranges cross from one
+    (batch, kv head) pair into the next."""
+    _full_size_case(oracle, 4, [(0, 0), (63, 3), (17, 2), (40, 1)], batch=64, seq=4096, n_q_heads=32, n_kv_heads=4,
+                    mant_bits=p)
 
 
 @pytest.mark.parametrize("p,impl", [(4, B.DECODE_AUTO), (8, B.DECODE_AUTO), (6, B.DECODE_AUTO), (4, B.DECODE_SIMT)])

@@ -35,16 +35,25 @@ def test_static_scratch_matches_regular_entry_point_twice():
 
     q1 = W.make_q(w, batch=Bn).cuda()
     q2 = (q1.float() * -0.5 + 0.25).to(q1.dtype)                 # a different query for the second call
-    cases = [(q1, [S, 301], B.DECODE_AUTO), (q2, [17, S], B.DECODE_SIMT)]
+    # the third call is much shorter than the ones before it: the array still holds their partial results in
+    # slots that this call's merge must not read
+    cases = [(q1, [S, 301], B.DECODE_AUTO), (q2, [17, S], B.DECODE_SIMT), (q1, [40, 0], B.DECODE_AUTO)]
     out = torch.empty(Bn, w.n_q_heads, 128, dtype=torch.float32, device="cuda")     # caller-owned output
-    for q, lens, impl in cases:
-        sl = torch.tensor(lens, dtype=torch.int32, device="cuda")
-        ref = B.decode_attn(cache, q, sl, perm_k=perm, impl=impl)
+    lens_dev = [torch.tensor(lens, dtype=torch.int32, device="cuda") for _, lens, _ in cases]
+    refs = [B.decode_attn(cache, q, sl, perm_k=perm, impl=impl) for (q, _, impl), sl in zip(cases, lens_dev)]
+    B.decode_attn_static(cache, q1, lens_dev[0], perm_k=perm, out=out)     # first call on the device: address look-up
+    torch.cuda.synchronize()
+    free0 = torch.cuda.mem_get_info()[0]
+    reserved0, allocated0 = torch.cuda.memory_reserved(), torch.cuda.memory_allocated()
+    for (q, lens, impl), sl, ref in zip(cases, lens_dev, refs):
         got = B.decode_attn_static(cache, q, sl, perm_k=perm, impl=impl, out=out)
         torch.cuda.synchronize()
         assert got.data_ptr() == out.data_ptr()
         assert rel_err(got, ref) <= ATTN_TOL
         assert torch.equal(got, ref)       # same kernels, same arithmetic: in fact identical
+    # nothing was allocated on the device by those calls, neither by the library nor through torch
+    assert torch.cuda.mem_get_info()[0] == free0
+    assert (torch.cuda.memory_reserved(), torch.cuda.memory_allocated()) == (reserved0, allocated0)
     assert B.device_status() == 0
 
 
