@@ -10,7 +10,7 @@
 // run's first chunk.  Each warp has a private ring of shared-memory stages filled by 1-D bulk
 // asynchronous copies (lanes 0..3 issue one span each, an mbarrier per stage counts the bytes); the
 // copies run ahead across run boundaries, so a new run starts with its first tiles already on chip.
-// There is no block-wide barrier in the loop and no cluster multicast.
+// There is no block-wide barrier in the loop; every warp fetches its own tiles.
 //
 // Unpacking is what limits this kernel (integer-pipe instructions, not memory).  A packed byte holds
 // two mantissas in excess-8 code: B = 16*(M_hi+8) + (M_lo+8).  fp16 path (P.V always; scores only for
@@ -54,26 +54,18 @@
 namespace kvbfp {
 namespace {
 
-#ifndef KVBFP4_WARPS
-#define KVBFP4_WARPS 4
-#endif
-#ifndef KVBFP4_MT
-#define KVBFP4_MT 4
-#endif
-#ifndef KVBFP4_STAGES
-#define KVBFP4_STAGES 2
-#endif
-#ifndef KVBFP4_MIN_CTAS
-#define KVBFP4_MIN_CTAS 3      // one 8-column tile; two tiles (groups of 5 to 8 heads) run two blocks per SM: with three
-#endif                         // they spill, and measured 9 % slower
-
-constexpr int kWarps = KVBFP4_WARPS;
-constexpr int kMT = KVBFP4_MT;          // 16-token MMA row tiles per stage
+constexpr int kWarps = 4;
+constexpr int kMT = 4;                  // 16-token MMA row tiles per stage
 constexpr int kTile = 16 * kMT;         // tokens per stage
-constexpr int kStages = KVBFP4_STAGES;
+constexpr int kStages = 2;
+constexpr int kMinCtas = 3;             // resident thread blocks per SM with one 8-column tile; two tiles (groups of 5 to
+                                        // 8 heads) run two blocks per SM: with three they spill, and measured 9 % slower
 constexpr int D = kHeadDim;
 constexpr int ROW_M = D / 2;            // 64 bytes of mantissas per token row
 constexpr int kTopShift = 5;            // weight of the run's largest block is 2^kTopShift
+constexpr int kTopShiftH = 7;           // the same in the single-head path, whose weights multiply the softmax weights
+                                        // (at most 2^8) before they are cut into fp16 halves: 2^15 at the most
+constexpr int kFlushStages = 4;         // single-head path: stages between two removals of the excess-code offsets
 constexpr int kDvHeadroom = 2;          // binades left above a tile's largest V exponent when the reference moves
 constexpr int kLutEntries = 512;        // index = exponent byte - D + 255, D = largest valid exponent byte
 
@@ -268,6 +260,109 @@ __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_
     }
 }
 
+// Single-head variant (one query head per kv head, blocks of 32 slots or more).  With one query the eight MMA
+// columns are free to separate the blocks instead of the queries: column 2*blk + digit holds the coefficient
+// digits of block blk and zeros elsewhere, so ONE accumulator set collects all blocks of a token and lane (g, t)
+// ends up with the two digit sums of (token g, block t).  The byte MMAs are 32 bytes deep; lane t feeds bytes
+// [16t, 16t + 16) of a token row: MMA j (0, 1) takes bytes 16t + 8j + (0..3) as k = 4t.., and 16t + 8j + 4 + (0..3)
+// as k = 16 + 4t...  The second operand of a packed word is the word shifted left by four bits WITHOUT a mask:
+// byte i of it is 16 * lo_i + hi_(i-1) (nothing for i = 0), still linear in the nibbles, so the two coefficient
+// rows a (whole byte) and b (shifted word) solve, per word and from its last byte down,
+//     16 a_i + b_(i+1) = q_hi_i,   a_i + 16 b_i = q_lo_i        (b_4 = 0)
+// and are cast to 15-bit fixed point with their block's exponent exactly like the coefficients above.
+// One warp per (batch, kv head).  qmeta[query][2 blk] = scale * log2(e) * 2^(qe - 16) (the factor 2^-2 of the
+// mantissa unit included), qmeta[query][2 blk + 1] = sum of 136 C (128 C for the shifted byte 0 of a word).
+__global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta) {
+    const int N = a.fmt.block, nblk = D / N, wpb = N / 8;       // wpb: 4-byte words per block
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gp = lane >> 2, tp = lane & 3;
+    const int item = blockIdx.x * 4 + warp;                     // (batch, kv head); one query head each
+    __shared__ float sq[4][D];
+    __shared__ int sC[4][2][D / 2];                             // [.][0]: whole-byte row a, [.][1]: shifted-word row b
+    if (item >= a.fmt.batch * a.fmt.n_kv_heads) return;
+    const int hk = item % a.fmt.n_kv_heads;
+    for (int i = lane; i < D; i += 32) {
+        const int ch = a.perm_k ? (a.perm_k[hk * D + i] & (D - 1)) : i;
+        const int64_t idx = (int64_t)item * D + ch;
+        sq[warp][i] = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
+    }
+    __syncwarp();
+    if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
+        if (lane < nblk) {
+            float* blk = &sq[warp][lane * N];
+            uint32_t am = 0;
+            for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(blk[j]) & 0x7fffffffu);
+            int e8 = (int)(am >> 23);
+            if (e8 == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e8 = 254; }
+            const int k = 127 - e8 + 6, k1 = k >> 1, k2 = k - k1;
+            const float w = unit_weight(e8, 8);
+            for (int j = 0; j < N; ++j) {
+                const float tv = (blk[j] * pow2i(k1)) * pow2i(k2);
+                blk[j] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * w;
+            }
+        }
+        __syncwarp();
+    }
+    // lanes 0..15 own one packed word each (bytes 4 lane .. 4 lane + 3 of the row)
+    float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
+    uint32_t am = 0;
+    if (lane < 16) {
+        float b_next = 0.f;
+#pragma unroll
+        for (int i = 3; i >= 0; --i) {
+            const int byte = 4 * lane + i;
+            ca[i] = (sq[warp][2 * byte + 1] - b_next) * 0.0625f;
+            cb[i] = (sq[warp][2 * byte] - ca[i]) * 0.0625f;
+            b_next = cb[i];
+            am = max(am, max(__float_as_uint(ca[i]) & 0x7fffffffu, __float_as_uint(cb[i]) & 0x7fffffffu));
+        }
+    }
+    for (int off = wpb >> 1; off; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+    int e = (int)(am >> 23);
+    if (e == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e = 254; }
+    const int qe = (am == 0) ? 0 : e - 126;                   // |c| * 2^-qe < 1
+    const int sh = 14 - qe, h1 = sh / 2, h2 = sh - h1;        // two exact factors (sh in [-114, 140])
+    int bias = 0;
+    if (lane < 16) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int Ca = __float2int_rn((ca[i] * pow2i(h1)) * pow2i(h2));
+            const int Cb = __float2int_rn((cb[i] * pow2i(h1)) * pow2i(h2));
+            sC[warp][0][4 * lane + i] = Ca;
+            sC[warp][1][4 * lane + i] = Cb;
+            bias += 136 * Ca + (i == 0 ? 128 : 136) * Cb;
+        }
+    }
+    for (int off = wpb >> 1; off; off >>= 1) bias += __shfl_xor_sync(0xffffffffu, bias, off);
+    int32_t* meta = qmeta + (int64_t)item * 8;
+    if (lane < 16 && lane % wpb == 0) {
+        meta[2 * (lane / wpb)] = __float_as_int(pow2_split(a.scale_log2e, qe - 16));
+        meta[2 * (lane / wpb) + 1] = bias;
+    }
+    if (lane >= 16 && lane < 16 + 4 - nblk) {                 // blocks that do not exist: factor 0, bias 0
+        meta[2 * (nblk + lane - 16)] = 0;
+        meta[2 * (nblk + lane - 16) + 1] = 0;
+    }
+    __syncwarp();
+    // fragments: word index 4 j + 2 kind + half (half 0: b0, k = 4t..; half 1: b1, k = 16 + 4t..)
+    const int cblk = gp >> 1, digit = gp & 1;
+    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
+#pragma unroll
+    for (int wd = 0; wd < 8; ++wd) {
+        const int j = wd >> 2, kind = (wd >> 1) & 1, half = wd & 1;
+        const int byte0 = 16 * tp + 8 * j + 4 * half;
+        uint32_t reg = 0;
+        if (byte0 / (N / 2) == cblk) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int C = sC[warp][kind][byte0 + i];
+                const int d1 = (C + 128) >> 8, d0 = C - 256 * d1;
+                reg |= ((uint32_t)(digit ? d0 : d1) & 0xffu) << (8 * i);
+            }
+        }
+        dst[((wd >> 2) * 32 + lane) * 4 + (wd & 3)] = reg;
+    }
+}
+
 // ------------------------------------------------------------------ main kernel
 template <int N>
 struct Geo4 {
@@ -322,13 +417,16 @@ __device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int la
     return (int)(m & 0xffu);
 }
 
-template <int N, int NT>
-__global__ void __launch_bounds__(kWarps * 32, NT == 1 ? KVBFP4_MIN_CTAS : 2) decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta) {
+// MHA: one query head per kv head and blocks of 32 slots or more -- the MMA columns separate the blocks of a row
+// instead of the query heads (see make_qfrag4h), in the scores and in P.V.
+template <int N, int NT, bool MHA>
+__global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta) {
     using G_ = Geo4<N>;
     constexpr int ROW_E = G_::ROW_E;
     constexpr int NBK = (N == 16) ? 2 : 1;            // blocks inside a K lane chunk of 32 slots
     constexpr bool KI = (N >= 32);                    // integer MMA path for the scores
     constexpr int NBLK = KI ? D / N : 1;              // blocks of a row (integer path)
+    static_assert(!MHA || (KI && NT == 1), "the single-head path is built on the integer scores");
     extern __shared__ __align__(128) uint8_t smem[];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;

@@ -5,7 +5,7 @@
 //
 // Same launch design as the 4-bit kernel: work items laid out pair-major and cut into one contiguous range per
 // resident warp (persistent), "runs" with one partial result each, a private ring of shared-memory stages per
-// warp filled by 1-D bulk asynchronous copies (no cluster multicast), no block-wide barrier in the loop.
+// warp filled by 1-D bulk asynchronous copies (each warp fetches its own tiles), no block-wide barrier in the loop.
 //
 // A stored byte is B = M + 128 (excess code), so nothing has to be unpacked.
 //   Scores: the bytes are the unsigned operand of a byte MMA.  The query block is cast to 15-bit fixed point

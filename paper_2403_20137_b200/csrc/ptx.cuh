@@ -1,5 +1,5 @@
 // Inline-PTX helpers shared by the tensor-core decode kernels: mbarrier + 1-D bulk asynchronous
-// copies (no cluster multicast), warp-level MMA, packed 16-bit arithmetic, byte permute, 3-input logic.
+// copies (one destination thread block each), warp-level MMA, packed 16-bit arithmetic, byte permute, 3-input logic.
 #pragma once
 #include <stdint.h>
 
@@ -119,6 +119,19 @@ __device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, 
 __device__ __forceinline__ void mma_u8s8_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t b0, int c_even, int c_odd) {
     asm("mma.sync.aligned.m16n8k16.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%8,%7,%8};"
         : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3]) : "r"(a0), "r"(a1), "r"(b0), "r"(c_even), "r"(c_odd));
+}
+// The same with 32 bytes per row: A = (a0: row g, k 4t..4t+3; a1: row g+8, same k; a2: row g, k 16+4t..; a3: row g+8),
+// B = (b0: k 4t..4t+3, column g; b1: k 16+4t.., column g).
+__device__ __forceinline__ void mma_u8s8_k32(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                             uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_u8s8_k32_first(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                   uint32_t b0, uint32_t b1, int c_even, int c_odd) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%10,%11};"
+        : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c_even), "r"(c_odd));
 }
 __device__ __forceinline__ uint32_t vmaxu4(uint32_t a, uint32_t b) { return __vmaxu4(a, b); }
 
