@@ -536,13 +536,25 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
         uint32_t qi8[NT][8];              // integer path: B fragments of the coefficient digits
         float qfac[NT][NBLK];             //   scale * log2(e) * 2^(qe - 14) per block
         int qbias[NT][NBLK];              //   offset contribution per block
+        float qfac_h = 0.f;               // single-head path: factor and offsets of this lane's block (block t)
+        int qbias_h = 0;
         {
             const uint4* src = reinterpret_cast<const uint4*>(a.qfrag);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
                 const int qn = 4 * nt + t;
                 const int32_t* meta = qmeta + ((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + (qn < Gq ? qn : 0)) * 8;
-                if (KI) {
+                if (MHA) {
+                    const uint4* s8 = src + ((int64_t)cr.b * Hkv + cr.hk) * (2 * 32);
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const uint4 v = __ldg(s8 + j * 32 + lane);
+                        qi8[0][4 * j] = v.x; qi8[0][4 * j + 1] = v.y; qi8[0][4 * j + 2] = v.z; qi8[0][4 * j + 3] = v.w;
+                    }
+                    const int32_t* mh = qmeta + ((int64_t)cr.b * Hkv + cr.hk) * 8;
+                    qfac_h = __int_as_float(mh[2 * t]);
+                    qbias_h = mh[2 * t + 1];
+                } else if (KI) {
                     const uint4* s8 = src + (((int64_t)cr.b * Hkv + cr.hk) * NT + nt) * (2 * 32);
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
@@ -575,6 +587,12 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
         int dv = 0;
         uint32_t dv_probe = 0x7FFF7FFFu;          // (0x7FFF - dv) in both halves: adding a byte > dv sets bit 15
         const uint2* lutv = lut + 255;
+        // single-head path: exponent byte e gives the fp32 weight 2^(e - dv + kTopShiftH) = bits (e + wexp) << 23;
+        // wsum collects this lane's weights (tokens g, g + 8 of every row tile, block t) since the last removal of
+        // the excess-code offsets from the sums
+        int wexp = 127 + kTopShiftH;
+        float wsum = 0.f;
+        int since_flush = 0;
         if (!KI) {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) kfac[nt] = pow2_split(a.scale_log2e, dk - 129 - kTopShift + (int)kfac[nt]);
@@ -619,7 +637,23 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                 dv = nd;
                 dv_probe = (0x7FFFu - (uint32_t)nd) * 0x00010001u;
                 lutv = lut + (255 - nd);
+                wexp = 127 + kTopShiftH - nd;
+                wsum *= f;
             }
+        };
+        // single-head path: the V bytes enter the MMAs as they are stored, so row "whole byte" carries 136 and row
+        // "low nibble" 8 per unit of weight too much; taken out of the hi-half column of the sums every few stages,
+        // while they are still small next to what they are taken from
+        auto flush_offsets = [&]() {
+            float w = wsum;
+            w += __shfl_xor_sync(0xffffffffu, w, 4);
+            w += __shfl_xor_sync(0xffffffffu, w, 8);
+            w += __shfl_xor_sync(0xffffffffu, w, 16);
+            const float c1 = w * (-136.f * 5.9604644775390625e-8f), c2 = w * (-8.f * 5.9604644775390625e-8f);   // 2^-24: the bytes are fp16 subnormals
+#pragma unroll
+            for (int r = 0; r < 8; ++r) { o[0][r][0] += c1; o[0][r][2] += c2; }
+            wsum = 0.f;
+            since_flush = 0;
         };
 
         // one stage of kTile tokens; FULL = every row of the tile exists
@@ -649,7 +683,29 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     for (int nt = 0; nt < NT; ++nt) sc[mt][nt][0] = sc[mt][nt][1] = -INFINITY;
                     continue;
                 }
-                if (KI) {
+                if (MHA) {
+                    // ---- single head: lane t feeds bytes [16t, 16t + 16) of tokens g and g + 8; the columns keep the
+                    // blocks apart, so all four MMAs go to one accumulator set
+                    const uint4 xa = *reinterpret_cast<const uint4*>(st + G_::KM_OFF + (mt * 16 + g) * ROW_M + 16 * t);
+                    const uint4 xb = *reinterpret_cast<const uint4*>(st + G_::KM_OFF + (mt * 16 + g + 8) * ROW_M + 16 * t);
+                    int acc[4];
+                    mma_u8s8_k32_first(acc, xa.x, xb.x, xa.y, xb.y, qi8[0][0], qi8[0][1], 0, -qbias_h);
+                    mma_u8s8_k32(acc, xa.z, xb.z, xa.w, xb.w, qi8[0][4], qi8[0][5]);
+                    mma_u8s8_k32(acc, xa.x << 4, xb.x << 4, xa.y << 4, xb.y << 4, qi8[0][2], qi8[0][3]);
+                    mma_u8s8_k32(acc, xa.z << 4, xb.z << 4, xa.w << 4, xb.w << 4, qi8[0][6], qi8[0][7]);
+                    // (256 * hi-digit sum + lo-digit sum) * 2^(e_k - 127) * (scale * 2^(qe - 16)) for block t, then the
+                    // four blocks of a token are added across the lanes t (an exponent byte of 0 counts as weight 0)
+                    constexpr int tb_mask = NBLK - 1;
+                    const uint32_t e0 = st[G_::KE_OFF + (mt * 16 + g) * ROW_E + (t & tb_mask)];
+                    const uint32_t e1 = st[G_::KE_OFF + (mt * 16 + g + 8) * ROW_E + (t & tb_mask)];
+                    float s0 = __int2float_rn(256 * acc[0] + acc[1]) * (__uint_as_float(e0 << 23) * qfac_h);
+                    float s1 = __int2float_rn(256 * acc[2] + acc[3]) * (__uint_as_float(e1 << 23) * qfac_h);
+                    s0 += __shfl_xor_sync(0xffffffffu, s0, 1);
+                    s1 += __shfl_xor_sync(0xffffffffu, s1, 1);
+                    s0 += __shfl_xor_sync(0xffffffffu, s0, 2);
+                    s1 += __shfl_xor_sync(0xffffffffu, s1, 2);
+                    sc[mt][0][0] = s0; sc[mt][0][1] = s1;
+                } else if (KI) {
                     // ---- integer path: bytes as they are (kind 1) and 16 x low nibble (kind 2), per 16-byte segment
                     int acc[NT][NBLK][4];
                     const uint8_t* pa = st + k_off + mt * 16 * ROW_M;
@@ -757,6 +813,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     const float alpha = (m_run[nt] == -INFINITY) ? 0.f : ex2_approx(m_run[nt] - m_new);
                     m_run[nt] = m_new;
                     l_run[nt] *= alpha;
+                    if (MHA) wsum *= alpha;
 #pragma unroll
                     for (int r = 0; r < 8; ++r)
 #pragma unroll
@@ -768,6 +825,48 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
 #pragma unroll
             for (int mt = 0; mt < kMT; ++mt) {
                 if (!FULL && mt * 16 >= n_live) continue;
+                if (MHA) {
+                    // ---- single head: the weight of (token, block t) = softmax weight x 2^(e_v - dv + kTopShiftH) is
+                    // formed here, in fp32, and travels as (hi, lo) fp16 halves in column (block, half); the V bytes
+                    // need no arithmetic at all: a byte under a zero exponent field is the fp16 subnormal byte * 2^-24
+                    constexpr int tb_mask = NBLK - 1;
+                    const float p0 = ex2_approx(sc[mt][0][0] - m_run[0]);
+                    const float p1 = ex2_approx(sc[mt][0][1] - m_run[0]);
+                    l_run[0] += p0 + p1;
+                    const int ev0 = st[G_::VE_OFF + (mt * 16 + g) * ROW_E + (t & tb_mask)];
+                    const int ev1 = st[G_::VE_OFF + (mt * 16 + g + 8) * ROW_E + (t & tb_mask)];
+                    float w0 = p0 * __int_as_float(max(ev0 + wexp, 0) << 23);
+                    float w1 = p1 * __int_as_float(max(ev1 + wexp, 0) << 23);
+                    if (!FULL) {       // rows past the end may hold any exponent byte: select, not arithmetic
+                        if (mt * 16 + g >= n_live) w0 = 0.f;
+                        if (mt * 16 + g + 8 >= n_live) w1 = 0.f;
+                    }
+                    wsum += w0 + w1;
+                    const float h0 = __uint_as_float(__float_as_uint(w0) & 0xffffe000u);
+                    const float h1 = __uint_as_float(__float_as_uint(w1) & 0xffffe000u);
+                    const uint32_t q0 = pack_f16x2_rn(h0, w0 - h0), q1 = pack_f16x2_rn(h1, w1 - h1);
+                    // B fragment for lane (g, t): column g = (block g/2, half g%2); tokens t, t+4 | t+8, t+12
+                    const uint32_t v0 = __shfl_sync(0xffffffffu, q0, src_lo);
+                    const uint32_t v1 = __shfl_sync(0xffffffffu, q0, src_hi);
+                    const uint32_t v2 = __shfl_sync(0xffffffffu, q1, src_lo);
+                    const uint32_t v3 = __shfl_sync(0xffffffffu, q1, src_hi);
+                    const uint32_t pb0 = prmt(v0, v1, half_sel), pb1 = prmt(v2, v3, half_sel);
+                    uint2 vw[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) vw[k] = *reinterpret_cast<const uint2*>(st + v_off + (mt * 16 + 4 * k) * ROW_M);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) {         // byte pair (2x, 2x+1) of the lane's eight bytes
+                        const uint32_t wA0 = (x < 2) ? vw[0].x : vw[0].y, wA1 = (x < 2) ? vw[1].x : vw[1].y;
+                        const uint32_t wB0 = (x < 2) ? vw[2].x : vw[2].y, wB1 = (x < 2) ? vw[3].x : vw[3].y;
+                        const uint32_t sel = (x & 1) ? 0x7632u : 0x5410u;
+                        const uint32_t XA = prmt(wA0, wA1, sel), XB = prmt(wB0, wB1, sel);     // [tok.b, tok.b', tok'.b, tok'.b']
+                        const uint32_t a1e = XA & 0x00FF00FFu, a1o = prmt(XA, 0u, 0x4341u);
+                        const uint32_t b1e = XB & 0x00FF00FFu, b1o = prmt(XB, 0u, 0x4341u);
+                        mma_f16(o[0][2 * x], a1e, XA & 0x000F000Fu, b1e, XB & 0x000F000Fu, pb0, pb1);
+                        mma_f16(o[0][2 * x + 1], a1o, a1o & 0x000F000Fu, b1o, b1o & 0x000F000Fu, pb0, pb1);
+                    }
+                    continue;
+                }
                 // softmax weights of this lane's tokens (g and g+8), then the B fragment of P^T for lane (g, t):
                 // column g = (query g/2, half g%2); tokens t, t+4 | t+8, t+12
                 uint32_t pb[NT][2];
@@ -833,6 +932,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
             const int n_live = cr.n_tok - it * kTile;        // tokens of this tile that exist (may exceed kTile)
             if (n_live >= kTile) tile_body(st, n_live, std::true_type{});
             else tile_body(st, n_live, std::false_type{});
+            if (MHA && ++since_flush == kFlushStages) flush_offsets();
             __syncwarp();
             issue_next(stage);
             if (++stage == kStages) { stage = 0; parity ^= 1u; }
@@ -841,6 +941,32 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
 
         // ---- partial result of the run, at the slot of its first chunk ----------------------------
         // row of kind 1 = 16*o_hi + o_lo, row of kind 2 = o_lo; common factor 2^(dv - 129 - kTopShift)
+        if (MHA) {
+            // lane (g, t) holds, for the bytes 8g..8g+7 of the row, the sums weighted for block t: the lanes whose t
+            // is the block of those bytes write them out.  2^24 undoes the subnormal scaling of the bytes.
+            flush_offsets();
+            const float vfac = pow2_split(1.f, dv - 129 - kTopShiftH);      // (2^24 apart: their product can leave the fp32 range)
+            const float vfac16 = vfac * 0.0625f;
+            float l = l_run[0];
+            l += __shfl_xor_sync(0xffffffffu, l, 4);
+            l += __shfl_xor_sync(0xffffffffu, l, 8);
+            l += __shfl_xor_sync(0xffffffffu, l, 16);
+            if (t == (16 * g) / N) {
+                float* dst = a.partials + (((int64_t)cr.b * a.n_q_heads + cr.hk) * a.n_chunks + partial_slot(cr.chunk0, a.item_tokens, a.chunk, a.n_chunks)) * kPartStride;
+#pragma unroll
+                for (int r4 = 0; r4 < 4; ++r4) {
+                    const float w0 = (o[0][2 * r4][0] + o[0][2 * r4][1]) * 16777216.f, l0 = (o[0][2 * r4][2] + o[0][2 * r4][3]) * 16777216.f;
+                    const float w1 = (o[0][2 * r4 + 1][0] + o[0][2 * r4 + 1][1]) * 16777216.f, l1 = (o[0][2 * r4 + 1][2] + o[0][2 * r4 + 1][3]) * 16777216.f;
+                    float4 v;
+                    v.x = l0 * vfac;            // slot 16g + 4r4     (low nibble of byte 2r4)
+                    v.y = (w0 - l0) * vfac16;   // slot 16g + 4r4 + 1 (high nibble of byte 2r4)
+                    v.z = l1 * vfac;
+                    v.w = (w1 - l1) * vfac16;
+                    reinterpret_cast<float4*>(dst + 16 * g)[r4] = v;
+                }
+                if (g == 0) { dst[D] = m_run[0]; dst[D + 1] = l; }
+            }
+        } else {
         const float vfac = pow2_split(1.f, dv - 129 - kTopShift);
         const float vfac16 = vfac * 0.0625f;
 #pragma unroll
@@ -866,6 +992,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                 if (g == 0) { dst[D] = m_run[nt]; dst[D + 1] = l; }
             }
         }
+        }
     }
 
     if (timed_out) {
@@ -878,7 +1005,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
     }
 }
 
-template <int N, int NT>
+template <int N, int NT, bool MHA>
 kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     using G_ = Geo4<N>;
     static std::atomic<int> resident[64];   // thread blocks that fit the whole device, per device (0 = not asked yet;
@@ -887,9 +1014,9 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     KVBFP_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return KVBFP_ERR_UNSUPPORTED;
     if (!resident[dev].load(std::memory_order_acquire)) {
-        KVBFP_CUDA(cudaFuncSetAttribute(decode_mma4<N, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_::SMEM_BYTES));
+        KVBFP_CUDA(cudaFuncSetAttribute(decode_mma4<N, NT, MHA>, cudaFuncAttributeMaxDynamicSharedMemorySize, G_::SMEM_BYTES));
         int per_sm = 0, n_sm = 0;
-        KVBFP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_mma4<N, NT>, kWarps * 32, G_::SMEM_BYTES));
+        KVBFP_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, decode_mma4<N, NT, MHA>, kWarps * 32, G_::SMEM_BYTES));
         KVBFP_CUDA(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
         if (per_sm < 1 || n_sm < 1) return KVBFP_ERR_CUDA;
         resident[dev].store(per_sm * n_sm, std::memory_order_release);
@@ -898,7 +1025,8 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     int32_t* qmeta = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
                                                (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
-    if (N >= 32) make_qfrag4i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
+    if (MHA) make_qfrag4h<<<(n_pre + 3) / 4, 128, 0, s>>>(a, qmeta);
+    else if (N >= 32) make_qfrag4i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
     else make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
     KVBFP_LAUNCH_CHECK("make_qfrag4");
     DecodeArgs b;
@@ -908,7 +1036,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma4<N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b, qmeta);
+    decode_mma4<N, NT, MHA><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b, qmeta);
     KVBFP_LAUNCH_CHECK("decode_mma4");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;
@@ -917,7 +1045,8 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
 template <int N>
 kvbfp_status launch2(const DecodeArgs& a, cudaStream_t s, Split* split) {
     const int G = a.n_q_heads / a.fmt.n_kv_heads;
-    return (G <= 4) ? launch3<N, 1>(a, s, split) : launch3<N, 2>(a, s, split);
+    if (N >= 32 && G == 1) return launch3<N, 1, (N >= 32)>(a, s, split);
+    return (G <= 4) ? launch3<N, 1, false>(a, s, split) : launch3<N, 2, false>(a, s, split);
 }
 
 }  // namespace
