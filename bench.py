@@ -260,6 +260,11 @@ def sweep_config5(B, dev):
     B.append(c, k, v, z, perm_k=perm)
     ms = timed(lambda: B.dequant(c, "k", 0, 0, 0, T, perm=perm), reps=5)
     out["dequant_one_head"] = {"tokens": T, "ms": ms, "GB/s": T * (68 + d * 4) / ms / 1e6}
+    for name, dt, eb in (("f32", torch.float32, 4), ("bf16", torch.bfloat16, 2)):
+        ms = timed(lambda: B.dequant_all(c, "k", T, perm=perm, out_dtype=dt), reps=5)
+        out[f"dequant_all_heads_{name}"] = {"tokens": T, "heads": H, "ms": ms, "GB/s": T * H * (68 + d * eb) / ms / 1e6}
+    ms = timed(lambda: B.dequant_all(c, "k", T), reps=5)
+    out["dequant_all_heads_f32_stored_order"] = {"tokens": T, "heads": H, "ms": ms, "GB/s": T * H * (68 + d * 4) / ms / 1e6}
     _, _, inv = B.calibrate(k[0, :4096].contiguous(), H, d)
     tabs = B.rope_tables(perm, inv, H, d, 10000.0, False, device=dev)
     rows = k[0]
@@ -282,6 +287,125 @@ def timed(fn, reps=1):
     return e0.elapsed_time(e1) / reps
 
 
+def kernel_name(B, w, impl):
+    if impl == B.DECODE_SIMT:
+        return "decode_simt"
+    if impl != B.DECODE_MMA_BF16 and w.mant_bits == 4:
+        return "decode_mma4"
+    if impl != B.DECODE_MMA_BF16 and w.mant_bits == 8 and w.block >= 32:
+        return "decode_mma8"
+    return "decode_mma"
+
+
+class StepRig:
+    """One configuration made resident on the device: calibrated permutation, a cache prefilled with S - 1 tokens per
+    sequence, the new token and the query of one decode step, output and workspace."""
+
+    def __init__(self, B, w, dev, impl, rope=False, chunk=0):
+        self.B, self.w, self.dev, self.impl, self.rope, self.chunk = B, w, dev, impl, rope, chunk
+        S, Bn, Hkv, Hq, d = w.seq, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim
+        self.es = 2 if w.dtype == "bf16" else 4
+        self.calib = W.make_calibration(w, device=dev)
+        _, self.perm_k, self.inv_perm_k = B.calibrate(self.calib, Hkv, d)
+        self.kernel = kernel_name(B, w, impl)
+        if rope:
+            self.impl, self.kernel = B.DECODE_SIMT, "decode_simt_rope"
+            self.rope_tabs = B.rope_tables(self.perm_k, self.inv_perm_k, Hkv, d, 10000.0, False, device=dev)
+        self.cache = B.Cache(Bn, Hkv, d, S, w.block, w.mant_bits, device=dev)
+        self.zeros = torch.zeros(Bn, dtype=torch.int32, device=dev)
+        k, v = W.make_kv(w, n_tokens=S, device=dev)                      # [B, S, Hkv, d]
+        self.k_pre, self.v_pre = k[:, :S - 1].contiguous(), v[:, :S - 1].contiguous()
+        B.append(self.cache, self.k_pre, self.v_pre, self.zeros, perm_k=self.perm_k)
+        self.k_new, self.v_new = k[:, S - 1:].contiguous(), v[:, S - 1:].contiguous()
+        del k, v
+        self.q = W.make_q(w, device=dev)
+        self.start_pos = torch.full((Bn,), S - 1, dtype=torch.int32, device=dev)
+        self.seq_lens = torch.full((Bn,), S, dtype=torch.int32, device=dev)
+        self.out = torch.empty(Bn, Hq, d, dtype=torch.float32, device=dev)
+        self.ws = torch.empty(B.decode_workspace_bytes(self.cache.fmt, Hq), dtype=torch.uint8, device=dev)
+        torch.cuda.synchronize()
+
+    def setup_timings(self):
+        """Set-up calls of the path, timed once (not part of the step metric)."""
+        B, w = self.B, self.w
+        ex = {}
+        ms = timed(lambda: B.calibrate(self.calib, w.n_kv_heads, w.head_dim), reps=3)
+        ex["calibrate"] = {"tokens": int(self.calib.shape[0]), "ms": ms, "GB/s": self.calib.numel() * self.es / ms / 1e6}
+        ms = timed(lambda: B.append(self.cache, self.k_pre, self.v_pre, self.zeros, perm_k=self.perm_k), reps=3)
+        rows = 2 * w.batch * (w.seq - 1) * w.n_kv_heads
+        row_bytes = w.head_dim * self.es + w.head_dim * w.mant_bits // 8 + w.head_dim // w.block
+        ex["append_prefill"] = {"tokens_per_seq": w.seq - 1, "ms": ms, "GB/s": rows * row_bytes / ms / 1e6,
+                                "elements/s": rows * w.head_dim / (ms * 1e-3)}
+        return ex
+
+    def free_setup(self):
+        del self.calib, self.k_pre, self.v_pre
+        self.calib = self.k_pre = self.v_pre = None
+
+    def step(self):
+        B, S = self.B, self.w.seq
+        B.append(self.cache, self.k_new, self.v_new, self.start_pos, perm_k=self.perm_k)
+        if self.rope:
+            B.decode_attn_rope(self.cache, self.q, self.seq_lens, *self.rope_tabs, perm_k=self.perm_k, max_len_hint=S,
+                               out=self.out, workspace=self.ws)
+        else:
+            B.decode_attn(self.cache, self.q, self.seq_lens, perm_k=self.perm_k, max_len_hint=S, impl=self.impl,
+                          out=self.out, workspace=self.ws, chunk_tokens=self.chunk)
+
+    def time_steps(self, steps, warmup, barrier):
+        """-> (ms of `steps` steps, launches): the timed region of the step metric, nothing but the steps in it."""
+        for _ in range(warmup):
+            self.step()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        launches0 = self.B.launch_count()
+        e0.record()
+        for _ in range(steps):
+            self.step()
+        e1.record()
+        barrier()
+        return e0.elapsed_time(e1), self.B.launch_count() - launches0
+
+    def time_kernel(self, steps, warmup, barrier):
+        """Mean duration (ms) of the main decode kernel over a second loop of the same steps, with a pair of CUDA
+        events recorded around that kernel on its own stream.  Kept apart from the loop that times the step, so
+        that the events sit in no step whose time is reported."""
+        B = self.B
+        kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, b in kev:              # an event gets its handle when it is first recorded
+            a.record()
+            b.record()
+        for _ in range(warmup):
+            self.step()
+        barrier()
+        for i in range(steps):
+            B.profile_decode_events(*kev[i])
+            self.step()
+        B.profile_decode_events(None, None)
+        barrier()
+        return statistics.mean(a.elapsed_time(b) for a, b in kev)
+
+
+def side_config(B, w, dev, impl, steps, warmup, local_rank, barrier):
+    """A further configuration in the default run: the same step (append 1 token + decode attention), timed the same
+    way, with its own clock sample.  -> dict for `extras`."""
+    rig = StepRig(B, w, dev, impl)
+    rig.free_setup()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    ms_total, _ = rig.time_steps(steps, warmup, barrier)
+    kernel_ms = rig.time_kernel(min(steps, 200), 3, barrier)
+    clocks = sampler.stop()
+    flags = B.device_status()
+    peak, _ = measured_peak()
+    alg = decode_bytes(w)
+    gbs = alg / (kernel_ms * 1e-3) / 1e9
+    return {"workload": workload_name(w), "decode_kernel": rig.kernel, "steps": steps, "ms_per_step": ms_total / steps,
+            "tokens/s": w.batch / (ms_total / steps * 1e-3), "kernel_ms": kernel_ms, "algorithmic_bytes": alg,
+            "GB/s": gbs, "frac_of_measured_peak": gbs / peak, "device_status_flags": flags, "clocks": clocks}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -300,9 +424,10 @@ def main():
     ap.add_argument("--block", type=int, default=0, choices=[0, 16, 32, 64, 128])
     ap.add_argument("--chunk", type=int, default=0, help="tokens per sequence chunk (0 = library default)")
     ap.add_argument("--rope", action="store_true", help="keys cached before the rotary embedding: time "
-                    "kvbfp_decode_attn_rope (fp32 kernel, rotation after the read-back) instead; no end-to-end leg")
+                    "kvbfp_decode_attn_rope (rotation after the read-back) instead; no end-to-end leg")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--no-extras", action="store_true", help="skip the set-up timings and the quality report")
+    ap.add_argument("--no-extras", action="store_true", help="skip the set-up timings, the quality report and the further "
+                    "configurations (GQA layer, mantissa sweep)")
     ap.add_argument("--sweep5", action="store_true", help="add the prefill/append and calibration sweep (8 KV heads, 65536 new\n                    tokens, blocks 16/32/64 x mantissas 4/6/8, calibration over 2^20 tokens) to the extras")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
@@ -329,111 +454,43 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
 
-    # ---- set-up (untimed for the step metric): calibrate, prefill S-1 tokens ----------------------
-    impl = {"auto": B.DECODE_AUTO, "simt": B.DECODE_SIMT, "mma": B.DECODE_MMA, "mma_bf16": B.DECODE_MMA_BF16}[args.decode_impl]
-    kernel = "decode_simt" if impl == B.DECODE_SIMT else \
-        ("decode_mma4" if (w.mant_bits == 4 and impl != B.DECODE_MMA_BF16) else
-         "decode_mma8" if (w.mant_bits == 8 and w.block >= 32 and impl != B.DECODE_MMA_BF16) else "decode_mma")
-    S, Bn, Hkv, Hq, d = w.seq, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim
-    es = 2 if w.dtype == "bf16" else 4
-    extras = {}
-    calib = W.make_calibration(w, device=dev)
-    _, perm_k, inv_perm_k = B.calibrate(calib, Hkv, d)
-    if args.rope:
-        impl, kernel, args.no_e2e = B.DECODE_SIMT, "decode_simt_rope", True
-        rope_tabs = B.rope_tables(perm_k, inv_perm_k, Hkv, d, 10000.0, False, device=dev)
-    if not args.no_extras:
-        ms = timed(lambda: B.calibrate(calib, Hkv, d), reps=3)
-        extras["calibrate"] = {"tokens": int(calib.shape[0]), "ms": ms, "GB/s": calib.numel() * es / ms / 1e6}
-    del calib
-    cache = B.Cache(Bn, Hkv, d, S, w.block, w.mant_bits, device=dev)
-    zeros = torch.zeros(Bn, dtype=torch.int32, device=dev)
-    k, v = W.make_kv(w, n_tokens=S, device=dev)                      # [B, S, Hkv, d]
-    k_pre, v_pre = k[:, :S - 1].contiguous(), v[:, :S - 1].contiguous()
-    B.append(cache, k_pre, v_pre, zeros, perm_k=perm_k)
-    if not args.no_extras:
-        ms = timed(lambda: B.append(cache, k_pre, v_pre, zeros, perm_k=perm_k), reps=3)
-        rows = 2 * Bn * (S - 1) * Hkv
-        row_bytes = d * es + d * w.mant_bits // 8 + d // w.block
-        extras["append_prefill"] = {"tokens_per_seq": S - 1, "ms": ms, "GB/s": rows * row_bytes / ms / 1e6,
-                                    "elements/s": rows * d / (ms * 1e-3)}
-        # quality on one head: key MSE and pre-softmax score error with and without K-sort (Table I's direction)
-        Tq = max(16, min(4096, (S - 1) // 16 * 16))
-        plain = B.Cache(1, Hkv, d, Tq, w.block, w.mant_bits, device=dev)
-        sortd = B.Cache(1, Hkv, d, Tq, w.block, w.mant_bits, device=dev)
-        z1 = torch.zeros(1, dtype=torch.int32, device=dev)
-        kk = k[:1, :Tq].contiguous()
-        B.append(plain, kk, None, z1)
-        B.append(sortd, kk, None, z1, perm_k=perm_k)
-        ref = kk[0, :, 0].float()
-        dq_p = B.dequant(plain, "k", 0, 0, 0, Tq)
-        dq_s = B.dequant(sortd, "k", 0, 0, 0, Tq, perm=perm_k)
-        qv = W.make_q(w, device=dev)[0, 0].float()
-        s_ref = ref @ qv
-        extras["quality_head0"] = {
-            "bits_per_element": w.mant_bits + 8.0 / w.block,
-            "key_mse_unsorted": float(((dq_p - ref) ** 2).mean()), "key_mse_ksort": float(((dq_s - ref) ** 2).mean()),
-            "score_rms_err_unsorted": float(((dq_p @ qv - s_ref) ** 2).mean().sqrt()),
-            "score_rms_err_ksort": float(((dq_s @ qv - s_ref) ** 2).mean().sqrt())}
-        del plain, sortd, kk, dq_p, dq_s
-    k_new, v_new = k[:, S - 1:].contiguous(), v[:, S - 1:].contiguous()
-    del k, v, k_pre, v_pre
-    if args.sweep5 and rank == 0:
-        extras["config5"] = sweep_config5(B, dev)
-    q = W.make_q(w, device=dev)
-    start_pos = torch.full((Bn,), S - 1, dtype=torch.int32, device=dev)
-    seq_lens = torch.full((Bn,), S, dtype=torch.int32, device=dev)
-    out = torch.empty(Bn, Hq, d, dtype=torch.float32, device=dev)
-    ws = torch.empty(B.decode_workspace_bytes(cache.fmt, Hq), dtype=torch.uint8, device=dev)
-    torch.cuda.synchronize()
-
-    def step():
-        B.append(cache, k_new, v_new, start_pos, perm_k=perm_k)
-        if args.rope:
-            B.decode_attn_rope(cache, q, seq_lens, *rope_tabs, perm_k=perm_k, max_len_hint=S, out=out, workspace=ws)
-        else:
-            B.decode_attn(cache, q, seq_lens, perm_k=perm_k, max_len_hint=S, impl=impl, out=out, workspace=ws,
-                          chunk_tokens=args.chunk)
-
     def barrier():
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing -------------------------------------------------------------------
-    for _ in range(args.warmup):
-        step()
-    kev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for a, b in kev:              # an event gets its handle when it is first recorded
-        a.record()
-        b.record()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # ---- set-up (untimed for the step metric): calibrate, prefill S-1 tokens ----------------------
+    impl = {"auto": B.DECODE_AUTO, "simt": B.DECODE_SIMT, "mma": B.DECODE_MMA, "mma_bf16": B.DECODE_MMA_BF16}[args.decode_impl]
+    S, Bn, Hkv, Hq, d = w.seq, w.batch, w.n_kv_heads, w.n_q_heads, w.head_dim
+    rig = StepRig(B, w, dev, impl, rope=args.rope, chunk=args.chunk)
+    if args.rope:
+        args.no_e2e = True
+    kernel, es = rig.kernel, rig.es
+    extras = {}
+    if not args.no_extras:
+        extras.update(rig.setup_timings())
+    rig.free_setup()
+    if args.sweep5 and rank == 0:
+        extras["config5"] = sweep_config5(B, dev)
+
+    # ---- device-resident timing: the step metric, then the main kernel's own duration ---------------
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    barrier()
-    launches0 = B.launch_count()
-    e0.record()
-    for i in range(args.steps):
-        B.profile_decode_events(*kev[i])
-        step()
-    e1.record()
-    barrier()
-    launches = B.launch_count() - launches0
-    B.profile_decode_events(None, None)
-    ms_total = e0.elapsed_time(e1)
-    kernel_ms = statistics.mean(a.elapsed_time(b) for a, b in kev)
+    ms_total, launches = rig.time_steps(args.steps, args.warmup, barrier)
+    kernel_steps = min(args.steps, 500)
+    kernel_ms = rig.time_kernel(kernel_steps, 3, barrier)
     flags = B.device_status()
 
     # ---- end to end: new token from pinned host memory, result back to the host, every step -------
-    hk, hv, hq = k_new.cpu().pin_memory(), v_new.cpu().pin_memory(), q.cpu().pin_memory()
+    hk, hv, hq = rig.k_new.cpu().pin_memory(), rig.v_new.cpu().pin_memory(), rig.q.cpu().pin_memory()
     hout = torch.empty(Bn, Hq, d, dtype=torch.float32).pin_memory()
-    staging = torch.empty(B.step_staging_bytes(cache.fmt, Hq, q.dtype), dtype=torch.uint8, device=dev)
+    staging = torch.empty(B.step_staging_bytes(rig.cache.fmt, Hq, rig.q.dtype), dtype=torch.uint8, device=dev)
 
     def step_host():
-        B.decode_step_host(cache, hk, hv, hq, start_pos, seq_lens, hout, staging, ws, perm_k=perm_k, max_len_hint=S,
-                           impl=impl)
+        B.decode_step_host(rig.cache, hk, hv, hq, rig.start_pos, rig.seq_lens, hout, staging, rig.ws, perm_k=rig.perm_k,
+                           max_len_hint=S, impl=rig.impl)
 
     n_e2e = 0 if args.no_e2e else args.steps
     for _ in range(args.warmup if n_e2e else 0):
@@ -447,7 +504,7 @@ def main():
     barrier()
     ms_e2e = f0.elapsed_time(f1) if n_e2e else float("nan")
     clocks = sampler.stop() if rank == 0 else None
-    e2e_ok = bool(torch.equal(hout.to(dev), out)) if n_e2e else None
+    e2e_ok = bool(torch.equal(hout.to(dev), rig.out)) if n_e2e else None
 
     # ---- max over ranks -----------------------------------------------------------------------------
     ms_total, ms_e2e, kernel_ms = max_over_ranks([ms_total, ms_e2e, kernel_ms], dist, dev)
@@ -455,6 +512,17 @@ def main():
         if dist is not None:
             dist.destroy_process_group()
         return
+
+    # ---- further configurations and the quality report (rank 0, outside every timed region above) ---
+    if not args.no_extras and world == 1 and not over and args.config == 3 and impl == B.DECODE_AUTO and not args.rope:
+        extras["config4"] = side_config(B, W.CONFIGS[4], dev, impl, 300, 10, local_rank, barrier)
+        extras["mant_sweep"] = {f"p{p}": side_config(B, dataclasses.replace(w, mant_bits=p), dev, impl, 300, 10,
+                                                     local_rank, barrier) for p in (6, 8)}
+    if not args.no_extras and world == 1:
+        from paper_2403_20137_b200 import quality as Q
+        nq = max(16, min(2048, S // 16 * 16))
+        extras["quality"] = Q.quality_report(w, dev, n_tokens=nq)
+        extras["quality_outliers_in_v"] = Q.quality_report(w, dev, n_tokens=nq, outliers_in_v=True, sort_v=True)
 
     ms_step = ms_total / args.steps
     value = whole_job_throughput(Bn, world, ms_step)
@@ -481,6 +549,8 @@ def main():
         "roofline": {"bound": "hbm", "kernel": kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "traffic": traffic_per_launch(kernel, w),
                      "algorithmic_bytes": alg, "kernel_ms": kernel_ms, "peak_source": peak_src,
+                     "kernel_timing": f"CUDA events around the main kernel, on its stream, in a loop of {kernel_steps} steps "
+                                      "of its own right after the loop that times the step",
                      "frac_of_nominal_8000_GBs": achieved / 8000.0},
         "extras": extras or None,
     }

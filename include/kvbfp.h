@@ -158,8 +158,13 @@ kvbfp_status kvbfp_append(const kvbfp_cache* cache, const void* k_new, const voi
 
 /*
  * Eq. (1): rows [t0, t0+n_tok) of (b, h) of one plane pair back to numbers (exact in f32 and bf16).
- *   perm  NULL: out[t, j] = slot j;  else out[t, perm[h*d+j]] = slot j (original channel order)
- *   out   [n_tok, head_dim] of out_dt
+ *   b, h  a sequence and a head, or -1 for all of them (one launch either way)
+ *   perm  [n_kv_heads*head_dim] i32 or NULL.  NULL: out[.., t, j] = slot j;
+ *         else out[.., t, perm[h*d+j]] = slot j (original channel order)
+ *   out   device, of out_dt: [n_tok, head_dim] for one (b, h); with h = -1 the heads come after the tokens,
+ *         [n_tok, n_kv_heads, head_dim]; with b = -1 the sequences come first, [batch, n_tok, ..] -- the layout
+ *         kvbfp_append takes its rows in
+ * Errors: rows past max_seq -> KVBFP_ERR_CAPACITY; nothing is written then.
  */
 kvbfp_status kvbfp_dequant(const kvbfp_format* fmt, const uint8_t* mant, const uint8_t* exp8,
                            int32_t b, int32_t h, int32_t t0, int32_t n_tok, const int32_t* perm,

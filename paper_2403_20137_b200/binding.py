@@ -228,6 +228,17 @@ def dequant(cache, which, b, h, t0, n_tok, perm=None, out_dtype=torch.float32, s
     return out
 
 
+def dequant_all(cache, which, n_tok, perm=None, t0=0, out_dtype=torch.float32, stream=None):
+    """kvbfp_dequant with b = h = -1: every sequence and head in one launch -> [B, n_tok, H_kv, d] of out_dtype
+    (the layout append() takes)."""
+    mant, exp8 = (cache.k_mant, cache.k_exp) if which == "k" else (cache.v_mant, cache.v_exp)
+    f = cache.fmt
+    out = torch.empty(f.batch, n_tok, f.n_kv_heads, f.head_dim, dtype=out_dtype, device=mant.device)
+    _check(lib().kvbfp_dequant(C.byref(f), _ptr(mant), _ptr(exp8), -1, -1, t0, n_tok,
+                               _ptr(_dev(perm, torch.int32)), _ptr(out), _dt(out), _stream(stream)))
+    return out
+
+
 def decode_workspace_bytes(fmt, n_q_heads):
     return int(lib().kvbfp_decode_workspace_bytes(C.byref(fmt), n_q_heads))
 

@@ -1,6 +1,7 @@
 // Shared host/device helpers of the kvbfp CUDA library (sm_100a).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -20,6 +21,12 @@ kvbfp_status status_word(uint32_t** ptr);
 void count_launch(int n = 1);
 // Number of SMs of the current device (asked once per device); grids are sized in multiples of it.
 kvbfp_status sm_count(int* n);
+
+// Tensor map over a plane of byte rows, [n_rows, row_bytes] (row_bytes 64 or 128), copied in boxes of box_rows whole
+// rows, swizzled in shared memory: the 16-byte pieces of a row land at piece ^ (row % 8) for rows of 128 bytes and at
+// piece ^ ((row / 2) % 4) for rows of 64 bytes, so that the same piece of eight neighbouring rows falls into eight
+// different bank groups.  The map covers memory of the current device only.
+kvbfp_status make_row_map(CUtensorMap* map, const void* base, uint64_t n_rows, uint32_t row_bytes, uint32_t box_rows);
 
 #define KVBFP_CUDA(call)                                                         \
     do {                                                                         \

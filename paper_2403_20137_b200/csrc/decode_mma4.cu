@@ -163,132 +163,35 @@ __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t*
     }
 }
 
-// Integer variant (blocks of 32 slots or more).  One 128-thread block per (batch, kv head, n-tile).  The coefficients of
-// every block are cast to C = round(c * 2^(14 - qe)) with the block's own exponent qe and written as two signed
-// byte digits, C = 256 * d1 + d0, in the B-fragment order of the byte MMA: fragment m = 2 * seg + kind covers the
-// bytes [16 seg, 16 seg + 16) of a row; lane (g, t) holds bytes 4t..4t+3 for column g = (query g/2, digit g%2:
-// 0 = d1, 1 = d0).  qmeta[query][2 blk] = scale * log2(e) * 2^(qe - 14) as float bits,
-// qmeta[query][2 blk + 1] = 136 * sum(C of kind 1) + 128 * sum(C of kind 2).
-__global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
-    // one thread per slot, the four query heads of the n-tile in turn; a block of 32 slots or more is made of whole
-    // warps, so block maxima and sums are reduced in the warp first
-    const int N = a.fmt.block, nblk = D / N;
-    const int s = threadIdx.x, blk = s / N;
-    const int item = blockIdx.x;
-    const int nt = item % NT, hk = (item / NT) % a.fmt.n_kv_heads, b = item / NT / a.fmt.n_kv_heads;
-    const int G = a.n_q_heads / a.fmt.n_kv_heads;
-    __shared__ int sC[4][D];              // fixed-point coefficients
-    __shared__ uint32_t smax[2][4][8];    // block maxima: [0] of q (BFP query cast), [1] of the coefficients
-    __shared__ int sbias[4][8];
-    if (s < 64) reinterpret_cast<uint32_t*>(smax)[s] = 0u;
-    if (s < 32) reinterpret_cast<int*>(sbias)[s] = 0;
-    __syncthreads();
-    const int ch = a.perm_k ? (a.perm_k[hk * D + s] & (D - 1)) : s;
-    float v[4];
-#pragma unroll
-    for (int qq = 0; qq < 4; ++qq) {
-        v[qq] = 0.f;
-        if (4 * nt + qq < G) {
-            const int64_t idx = ((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * D + ch;
-            v[qq] = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
-        }
-    }
-    if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
-#pragma unroll
-        for (int qq = 0; qq < 4; ++qq) {
-            const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(v[qq]) & 0x7fffffffu);
-            if ((s & 31) == 0) atomicMax(&smax[0][qq][blk], mx);
-        }
-        __syncthreads();
-#pragma unroll
-        for (int qq = 0; qq < 4; ++qq) {
-            int e8 = (int)(smax[0][qq][blk] >> 23);
-            if (e8 == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e8 = 254; }
-            const int k = 127 - e8 + 6, k1 = k >> 1, k2 = k - k1;
-            const float tv = (v[qq] * pow2i(k1)) * pow2i(k2);
-            v[qq] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * unit_weight(e8, 8);
-        }
-    }
-    // coefficients: odd slot 2j+1 <- c1 = q_hi/16 (kind 1: whole byte), even slot 2j <- c2 = (q_lo - q_hi/16)/16
-    // (kind 2: 16 x low nibble).  Both multiply operands that carry a factor 16, so they have the same size and
-    // one block exponent serves both without losing bits of either.
-    float c[4];
-#pragma unroll
-    for (int qq = 0; qq < 4; ++qq) {
-        const float other = __shfl_xor_sync(0xffffffffu, v[qq], 1);
-        c[qq] = (s & 1) ? v[qq] * 0.0625f : (v[qq] - other * 0.0625f) * 0.0625f;
-        const uint32_t mx = __reduce_max_sync(0xffffffffu, __float_as_uint(c[qq]) & 0x7fffffffu);
-        if ((s & 31) == 0) atomicMax(&smax[1][qq][blk], mx);
-    }
-    __syncthreads();
-#pragma unroll
-    for (int qq = 0; qq < 4; ++qq) {
-        const uint32_t am = smax[1][qq][blk];
-        int e = (int)(am >> 23);
-        if (e == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e = 254; }
-        const int qe = (am == 0) ? 0 : e - 126;               // |c| * 2^-qe < 1
-        const int sh = 14 - qe, h1 = sh / 2, h2 = sh - h1;    // two exact factors (sh in [-114, 140])
-        const int C = __float2int_rn((c[qq] * pow2i(h1)) * pow2i(h2));
-        sC[qq][s] = C;
-        const int bsum = __reduce_add_sync(0xffffffffu, ((s & 1) ? 136 : 128) * C);
-        if ((s & 31) == 0) atomicAdd(&sbias[qq][blk], bsum);
-        if (s % N == 0 && 4 * nt + qq < G)
-            qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * blk] = __float_as_int(pow2_split(a.scale_log2e, qe - 14));
-    }
-    __syncthreads();
-    if (s < 4 * nblk) {
-        const int qq = s / nblk, k = s % nblk;
-        if (4 * nt + qq < G) qmeta[((int64_t)b * a.n_q_heads + hk * G + 4 * nt + qq) * 8 + 2 * k + 1] = sbias[qq][k];
-    }
-    // fragments: word (m, lane) for m = 0..7; thread s writes (m = s / 32, lane = s % 32) and (m + 4, lane)
-    const int lane = s & 31, gp = lane >> 2, tp = lane & 3;
-    const int qq = gp >> 1, digit = gp & 1, qi = 4 * nt + qq;
-    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
-#pragma unroll
-    for (int mm = 0; mm < 2; ++mm) {
-        const int m = (s >> 5) + 4 * mm, seg = m >> 1, kind = m & 1;
-        uint32_t reg = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int byte = 16 * seg + 4 * tp + e;
-            const int C = sC[qq][2 * byte + (kind == 0 ? 1 : 0)];
-            const int d1 = (C + 128) >> 8, d0 = C - 256 * d1;
-            const int dsel = (qi < G) ? (digit ? d0 : d1) : 0;
-            reg |= ((uint32_t)dsel & 0xffu) << (8 * e);
-        }
-        dst[((m >> 2) * 32 + lane) * 4 + (m & 3)] = reg;
-    }
-}
-
-// Single-head variant (one query head per kv head, blocks of 32 slots or more).  With one query the eight MMA
-// columns are free to separate the blocks instead of the queries: column 2*blk + digit holds the coefficient
-// digits of block blk and zeros elsewhere, so ONE accumulator set collects all blocks of a token and lane (g, t)
-// ends up with the two digit sums of (token g, block t).  The byte MMAs are 32 bytes deep; lane t feeds bytes
-// [16t, 16t + 16) of a token row: MMA j (0, 1) takes bytes 16t + 8j + (0..3) as k = 4t.., and 16t + 8j + 4 + (0..3)
-// as k = 16 + 4t...  The second operand of a packed word is the word shifted left by four bits WITHOUT a mask:
-// byte i of it is 16 * lo_i + hi_(i-1) (nothing for i = 0), still linear in the nibbles, so the two coefficient
-// rows a (whole byte) and b (shifted word) solve, per word and from its last byte down,
+// ---- integer scores (blocks of 32 slots or more) --------------------------------------------------------------
+// The K bytes enter unsigned-byte x signed-byte MMAs twice: as they are, and as the packed 32-bit word shifted left
+// by four bits WITHOUT a mask: byte i of that is 16 * lo_i + hi_(i-1) (nothing for i = 0), still linear in the
+// nibbles.  The two coefficient rows a (whole byte) and b (shifted word) therefore solve, per word and from its last
+// byte down,
 //     16 a_i + b_(i+1) = q_hi_i,   a_i + 16 b_i = q_lo_i        (b_4 = 0)
-// and are cast to 15-bit fixed point with their block's exponent exactly like the coefficients above.
-// One warp per (batch, kv head).  qmeta[query][2 blk] = scale * log2(e) * 2^(qe - 16) (the factor 2^-2 of the
-// mantissa unit included), qmeta[query][2 blk + 1] = sum of 136 C (128 C for the shifted byte 0 of a word).
-__global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta) {
-    const int N = a.fmt.block, nblk = D / N, wpb = N / 8;       // wpb: 4-byte words per block
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gp = lane >> 2, tp = lane & 3;
-    const int item = blockIdx.x * 4 + warp;                     // (batch, kv head); one query head each
-    __shared__ float sq[4][D];
-    __shared__ int sC[4][2][D / 2];                             // [.][0]: whole-byte row a, [.][1]: shifted-word row b
-    if (item >= a.fmt.batch * a.fmt.n_kv_heads) return;
-    const int hk = item % a.fmt.n_kv_heads;
+// They are cast to 15-bit fixed point, C = round(c * 2^(14 - qe)), with the exponent qe of their block and written as
+// two signed byte digits, C = 256 * d1 + d0, which sit in two MMA columns; the two 32-bit sums of a (token, block) are
+// recombined exactly, the constant contribution of the excess-8 offsets (136 per whole byte, 136 per shifted byte
+// but 128 for byte 0 of a word) goes into the accumulator beforehand, and one fp32 multiply-add applies
+// 2^(e_k - 127) * scale * log2(e) * 2^(qe - 16) per (token, block) (the factor 2^-2 of the mantissa unit included).
+
+// One warp, one query head: pi(q) -> sq[D]; with q_mant_bits the BFP16 cast of Sec. IV (blocks of N slots, 8-bit
+// mantissas) in place.
+__device__ __forceinline__ void load_query_row(const DecodeArgs& a, int64_t q_row, int hk, bool live, int lane, float* sq) {
+    const int N = a.fmt.block;
     for (int i = lane; i < D; i += 32) {
-        const int ch = a.perm_k ? (a.perm_k[hk * D + i] & (D - 1)) : i;
-        const int64_t idx = (int64_t)item * D + ch;
-        sq[warp][i] = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
+        float v = 0.f;
+        if (live) {
+            const int ch = a.perm_k ? (a.perm_k[hk * D + i] & (D - 1)) : i;
+            const int64_t idx = q_row * D + ch;
+            v = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
+        }
+        sq[i] = v;
     }
     __syncwarp();
-    if (a.q_mant_bits) {   // BFP query (Sec. IV): blocks of N slots, 8-bit mantissas
-        if (lane < nblk) {
-            float* blk = &sq[warp][lane * N];
+    if (a.q_mant_bits) {
+        if (lane < D / N) {
+            float* blk = &sq[lane * N];
             uint32_t am = 0;
             for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(blk[j]) & 0x7fffffffu);
             int e8 = (int)(am >> 23);
@@ -302,7 +205,13 @@ __global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta
         }
         __syncwarp();
     }
-    // lanes 0..15 own one packed word each (bytes 4 lane .. 4 lane + 3 of the row)
+}
+// One warp, one query head: the coefficient rows of sq[D] as fixed-point integers, sCa[byte] (whole byte) and
+// sCb[byte] (shifted word), and per block meta[2 blk] = scale * log2(e) * 2^(qe - 16) as float bits,
+// meta[2 blk + 1] = the offsets' contribution (meta == nullptr: not written).  Lanes 0..15 own one packed word each
+// (bytes 4 lane .. 4 lane + 3 of the row).
+__device__ __forceinline__ void coefficient_rows(const DecodeArgs& a, const float* sq, int lane, int* sCa, int* sCb, int32_t* meta) {
+    const int N = a.fmt.block, nblk = D / N, wpb = N / 8;       // wpb: 4-byte words per block
     float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
     uint32_t am = 0;
     if (lane < 16) {
@@ -310,8 +219,8 @@ __global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta
 #pragma unroll
         for (int i = 3; i >= 0; --i) {
             const int byte = 4 * lane + i;
-            ca[i] = (sq[warp][2 * byte + 1] - b_next) * 0.0625f;
-            cb[i] = (sq[warp][2 * byte] - ca[i]) * 0.0625f;
+            ca[i] = (sq[2 * byte + 1] - b_next) * 0.0625f;
+            cb[i] = (sq[2 * byte] - ca[i]) * 0.0625f;
             b_next = cb[i];
             am = max(am, max(__float_as_uint(ca[i]) & 0x7fffffffu, __float_as_uint(cb[i]) & 0x7fffffffu));
         }
@@ -327,22 +236,74 @@ __global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta
         for (int i = 0; i < 4; ++i) {
             const int Ca = __float2int_rn((ca[i] * pow2i(h1)) * pow2i(h2));
             const int Cb = __float2int_rn((cb[i] * pow2i(h1)) * pow2i(h2));
-            sC[warp][0][4 * lane + i] = Ca;
-            sC[warp][1][4 * lane + i] = Cb;
+            sCa[4 * lane + i] = Ca;
+            sCb[4 * lane + i] = Cb;
             bias += 136 * Ca + (i == 0 ? 128 : 136) * Cb;
         }
     }
     for (int off = wpb >> 1; off; off >>= 1) bias += __shfl_xor_sync(0xffffffffu, bias, off);
-    int32_t* meta = qmeta + (int64_t)item * 8;
-    if (lane < 16 && lane % wpb == 0) {
-        meta[2 * (lane / wpb)] = __float_as_int(pow2_split(a.scale_log2e, qe - 16));
-        meta[2 * (lane / wpb) + 1] = bias;
-    }
-    if (lane >= 16 && lane < 16 + 4 - nblk) {                 // blocks that do not exist: factor 0, bias 0
-        meta[2 * (nblk + lane - 16)] = 0;
-        meta[2 * (nblk + lane - 16) + 1] = 0;
+    if (meta) {
+        if (lane < 16 && lane % wpb == 0) {
+            meta[2 * (lane / wpb)] = __float_as_int(pow2_split(a.scale_log2e, qe - 16));
+            meta[2 * (lane / wpb) + 1] = bias;
+        }
+        if (lane >= 16 && lane < 16 + 4 - nblk) {                 // blocks that do not exist: factor 0, bias 0
+            meta[2 * (nblk + lane - 16)] = 0;
+            meta[2 * (nblk + lane - 16) + 1] = 0;
+        }
     }
     __syncwarp();
+}
+
+// Several query heads per kv head.  One 128-thread block per (batch, kv head, n-tile), one warp per query head of the
+// n-tile.  B fragments of the 32-byte-deep MMAs: word 2 * seg + kind covers the bytes [16 seg, 16 seg + 16) of a row
+// (kind 0: whole bytes, kind 1: shifted words); lane (g, t) holds bytes 4t..4t+3 for column g = (query g/2, digit
+// g%2: 0 = d1, 1 = d0).
+__global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gp = lane >> 2, tp = lane & 3;
+    const int item = blockIdx.x;
+    const int nt = item % NT, hk = (item / NT) % a.fmt.n_kv_heads, b = item / NT / a.fmt.n_kv_heads;
+    const int G = a.n_q_heads / a.fmt.n_kv_heads;
+    __shared__ float sq[4][D];
+    __shared__ int sC[4][2][D / 2];                             // [.][0]: whole-byte row a, [.][1]: shifted-word row b
+    const int qi_w = 4 * nt + warp;                             // this warp's query head within the group
+    const int64_t q_row = (int64_t)b * a.n_q_heads + hk * G + qi_w;
+    load_query_row(a, q_row, hk, qi_w < G, lane, sq[warp]);
+    coefficient_rows(a, sq[warp], lane, sC[warp][0], sC[warp][1], qi_w < G ? qmeta + q_row * 8 : nullptr);
+    __syncthreads();
+    // fragments: word (m, lane) for m = 0..7; thread s writes (m = s / 32, lane) and (m + 4, lane)
+    const int qq = gp >> 1, digit = gp & 1, qi = 4 * nt + qq;
+    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
+#pragma unroll
+    for (int mm = 0; mm < 2; ++mm) {
+        const int m = warp + 4 * mm, seg = m >> 1, kind = m & 1;
+        uint32_t reg = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int C = sC[qq][kind][16 * seg + 4 * tp + e];
+            const int d1 = (C + 128) >> 8, d0 = C - 256 * d1;
+            const int dsel = (qi < G) ? (digit ? d0 : d1) : 0;
+            reg |= ((uint32_t)dsel & 0xffu) << (8 * e);
+        }
+        dst[((m >> 2) * 32 + lane) * 4 + (m & 3)] = reg;
+    }
+}
+
+// One query head per kv head.  With one query the eight MMA columns are free to separate the blocks instead of the
+// queries: column 2*blk + digit holds the coefficient digits of block blk and zeros elsewhere, so ONE accumulator set
+// collects all blocks of a token and lane (g, t) ends up with the two digit sums of (token g, block t).  Lane t feeds
+// bytes [16t, 16t + 16) of a token row: MMA j (0, 1) takes bytes 16t + 8j + (0..3) as k = 4t.., and
+// 16t + 8j + 4 + (0..3) as k = 16 + 4t...  One warp per (batch, kv head).
+__global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta) {
+    const int N = a.fmt.block;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gp = lane >> 2, tp = lane & 3;
+    const int item = blockIdx.x * 4 + warp;                     // (batch, kv head); one query head each
+    __shared__ float sq[4][D];
+    __shared__ int sC[4][2][D / 2];                             // [.][0]: whole-byte row a, [.][1]: shifted-word row b
+    if (item >= a.fmt.batch * a.fmt.n_kv_heads) return;
+    const int hk = item % a.fmt.n_kv_heads;
+    load_query_row(a, item, hk, true, lane, sq[warp]);
+    coefficient_rows(a, sq[warp], lane, sC[warp][0], sC[warp][1], qmeta + (int64_t)item * 8);
     // fragments: word index 4 j + 2 kind + half (half 0: b0, k = 4t..; half 1: b1, k = 16 + 4t..)
     const int cblk = gp >> 1, digit = gp & 1;
     uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
@@ -364,20 +325,34 @@ __global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta
 }
 
 // ------------------------------------------------------------------ main kernel
+// Shared memory of a thread block.  The mantissa tiles come first: every (warp, stage) has a K tile and a V tile of
+// kTile token rows x 64 bytes, each 4 KiB and aligned to 1 KiB.  They are filled by tiled 2-D copies that take the
+// plane as rows of 128 bytes (two tokens: whole 128-byte lines move) and swizzle the 16-byte pieces of such a row,
+// piece ^ (row % 8): token rows are 64 bytes apart, so without it the same piece of tokens g and g + 2 would sit in the
+// same banks.  Exponent bytes, the weight table and the barriers follow.
+constexpr int kTileBytes = kTile * ROW_M;
 template <int N>
 struct Geo4 {
     static constexpr int ROW_E = D / N;
+    static constexpr int MANT_STAGE = 2 * kTileBytes;                   // K tile, V tile
     static constexpr int KM_OFF = 0;
-    static constexpr int VM_OFF = kTile * ROW_M;
-    static constexpr int KE_OFF = 2 * kTile * ROW_M;
-    static constexpr int VE_OFF = KE_OFF + kTile * ROW_E;
-    static constexpr int STAGE_BYTES = 2 * kTile * (ROW_M + ROW_E);
-    static constexpr int WARP_BYTES = kStages * STAGE_BYTES;
-    static constexpr int LUT_OFF = kWarps * WARP_BYTES;                 // uint2[kLutEntries]
-    static constexpr int LUTF_OFF = LUT_OFF + kLutEntries * 8;          // float[256] (integer score path)
-    static constexpr int BAR_OFF = LUTF_OFF + (N >= 32 ? 256 * 4 : 0);
+    static constexpr int VM_OFF = kTileBytes;
+    static constexpr int EXP_OFF = kWarps * kStages * MANT_STAGE;       // per (warp, stage): K bytes, V bytes
+    static constexpr int EXP_STAGE = 2 * kTile * ROW_E;
+    static constexpr int KE_OFF = 0;
+    static constexpr int VE_OFF = kTile * ROW_E;
+    static constexpr int LUT_OFF = EXP_OFF + kWarps * kStages * EXP_STAGE;   // uint2[kLutEntries]
+    static constexpr int BAR_OFF = LUT_OFF + kLutEntries * 8;
     static constexpr int SMEM_BYTES = BAR_OFF + kWarps * kStages * 8;
 };
+// Offset of 16-byte piece `piece` (0..3) of token row `tok` inside a swizzled tile.
+__device__ __forceinline__ int swz(int tok, int piece) {
+    return (tok >> 1) * 128 + (((4 * (tok & 1) + piece) ^ ((tok >> 1) & 7)) << 4);
+}
+// P.V: lane column t holds tokens tok4(t, 0..3) of a 16-token row tile as the k positions (2t, 2t+1, 2t+8, 2t+9) of the
+// MMA.  Which tokens is free (the softmax weights are brought along); these make the 8-byte V loads of a half warp
+// (tokens tok4(0..3, k), pieces 0 and 1 or 2 and 3) fall into distinct banks of the swizzled tile.
+__host__ __device__ constexpr int tok4(int t, int k) { return (t & 1) + 4 * (t >> 1) + 2 * (k & 1) + 8 * (k >> 1); }
 
 // Largest of the first `bytes` bytes of a 16-byte-aligned span in global memory, over the warp.  Whole
 // 16-byte vectors are loaded (the span is padded to a multiple of 16 inside the plane); bytes past
@@ -420,14 +395,16 @@ __device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int la
 // MHA: one query head per kv head and blocks of 32 slots or more -- the MMA columns separate the blocks of a row
 // instead of the query heads (see make_qfrag4h), in the scores and in P.V.
 template <int N, int NT, bool MHA>
-__global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta) {
+__global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2)
+decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_constant__ CUtensorMap k_map,
+            const __grid_constant__ CUtensorMap v_map) {
     using G_ = Geo4<N>;
     constexpr int ROW_E = G_::ROW_E;
     constexpr int NBK = (N == 16) ? 2 : 1;            // blocks inside a K lane chunk of 32 slots
     constexpr bool KI = (N >= 32);                    // integer MMA path for the scores
     constexpr int NBLK = KI ? D / N : 1;              // blocks of a row (integer path)
     static_assert(!MHA || (KI && NT == 1), "the single-head path is built on the integer scores");
-    extern __shared__ __align__(128) uint8_t smem[];
+    extern __shared__ __align__(1024) uint8_t smem[];         // the swizzle pattern is a function of the address
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
@@ -458,8 +435,13 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
         return r;
     };
 
-    uint8_t* wsm = smem + warp * G_::WARP_BYTES;
-    const uint32_t wsm_u32 = smem_u32(wsm);
+    if (smem_u32(smem) & 1023u) {        // never expected: the tiles would be read with the wrong pattern
+        if (threadIdx.x == 0) raise_flag(a.status, KVBFP_FLAG_WAIT_TIMEOUT);
+        return;                          // (the whole block, before any copy is issued)
+    }
+    uint8_t* wsm = smem + warp * kStages * G_::MANT_STAGE;                          // this warp's mantissa tiles
+    uint8_t* wse = smem + G_::EXP_OFF + warp * kStages * G_::EXP_STAGE;             // and exponent bytes
+    const uint32_t wsm_u32 = smem_u32(wsm), wse_u32 = smem_u32(wse);
     const uint32_t bar0 = smem_u32(smem + G_::BAR_OFF + warp * kStages * 8);
     if (lane == 0) {
 #pragma unroll
@@ -469,11 +451,14 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
     }
     __syncwarp();
 
-    // ---- producer: lanes 0..3 each own one of the four spans of a stage (K mantissas, V mantissas,
-    // K exponents, V exponents).  The cursor (p_run, p_tile) runs ahead of the consumer by kStages tiles.
-    const uint8_t* my_base = lane == 0 ? a.k_mant : lane == 1 ? a.v_mant : lane == 2 ? a.k_exp : a.v_exp;
-    const int my_row_bytes = (lane < 2) ? ROW_M : ROW_E;
-    const uint32_t my_dst = wsm_u32 + (lane == 0 ? G_::KM_OFF : lane == 1 ? G_::VM_OFF : lane == 2 ? G_::KE_OFF : G_::VE_OFF);
+    // ---- producer: lanes 0..3 each own one of the four pieces of a stage: the K and V mantissa tiles (tiled copies of
+    // kTile whole rows: rows past the sequence are never used, rows past the plane arrive as zeros) and the K and V
+    // exponent bytes (1-D copies of the 16-token groups that hold tokens).  The cursor (p_run, p_tile) runs ahead of
+    // the consumer by kStages tiles.
+    const uint8_t* my_exp = lane == 2 ? a.k_exp : a.v_exp;
+    const CUtensorMap* my_map = lane == 0 ? &k_map : &v_map;
+    const uint32_t my_dst = lane < 2 ? wsm_u32 + (lane == 0 ? G_::KM_OFF : G_::VM_OFF)
+                                     : wse_u32 + (lane == 2 ? G_::KE_OFF : G_::VE_OFF);
     int p_next = i0;
     Run pr;
     pr.n_tiles = 0;
@@ -489,36 +474,44 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
             const int off = p_tile * kTile;
             const int rows = min(kTile, ((pr.n_tok + 15) & ~15) - off);    // whole 16-token groups; stays below max_seq
             const uint32_t bar = bar0 + 8 * stage;
-            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(2 * rows * (ROW_M + ROW_E)));
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(2 * kTileBytes + 2 * rows * ROW_E));
             __syncwarp(0xfu);
-            bulk_g2s(my_dst + stage * G_::STAGE_BYTES, my_base + (pr.row0 + off) * my_row_bytes, rows * my_row_bytes, bar);
+            if (lane < 2) tensor_g2s_2d(my_dst + stage * G_::MANT_STAGE, my_map, 0, (int)((pr.row0 + off) >> 1), bar);
+            else bulk_g2s(my_dst + stage * G_::EXP_STAGE, my_exp + (pr.row0 + off) * ROW_E, rows * ROW_E, bar);
         }
         ++p_tile;
     };
     for (int s = 0; s < kStages; ++s) issue_next(s);
 
-    // (the tables are filled while the first copies are in flight)
+    // (the table is filled while the first copies are in flight)
     // weight table: entry i = (2^(i - 255 + kTopShift) twice as f16x2, the same times -1160); entries
     // above 255 belong to rows that are masked later (past the end of the run) and only have to exist
     uint2* lut = reinterpret_cast<uint2*>(smem + G_::LUT_OFF);
-    for (int i = threadIdx.x; i < kLutEntries; i += kWarps * 32) {
-        const uint32_t s2 = (i <= 255 ? pow2_f16(i - 255 + kTopShift) : 0u) * 0x00010001u;
-        lut[i] = make_uint2(s2, mul_f16x2(s2, kBias));
-    }
-    // integer score path: 2^(e - 129), the true weight of a mantissa unit, as fp32 (no range issue there)
-    float* lutf = reinterpret_cast<float*>(smem + G_::LUTF_OFF);
-    if (KI)
-        for (int i = threadIdx.x; i < 256; i += kWarps * 32) lutf[i] = unit_weight(i, 4);
+    if (!MHA)
+        for (int i = threadIdx.x; i < kLutEntries; i += kWarps * 32) {
+            const uint32_t s2 = (i <= 255 ? pow2_f16(i - 255 + kTopShift) : 0u) * 0x00010001u;
+            lut[i] = make_uint2(s2, mul_f16x2(s2, kBias));
+        }
     __syncthreads();
     if (i0 >= i1) return;
 
-    // per-lane byte offsets inside a stage
-    const int k_off = G_::KM_OFF + g * ROW_M + t * (KI ? 4 : 16);
+    // per-lane byte offsets inside a stage (mantissa tiles swizzled, see Geo4)
+    const int k_off = G_::KM_OFF + swz(g, t);                  // 16 bytes [16t, 16t + 16) of token g,
+    const int k_off8 = G_::KM_OFF + swz(g + 8, t);             // of token g + 8
+    // integer scores with several query heads: addresses for the 8 x 16-byte matrix loads.  Lane i names row i % 8 of
+    // matrix i / 8; matrices 0, 1 = rows 0..7 and 8..15 of 16-byte piece 0 (piece 2 with the address bit 5 flipped),
+    // matrices 2, 3 = the same rows of piece 1 (3)
+    const int lm_off = G_::KM_OFF + swz(8 * ((lane >> 3) & 1) + (lane & 7), lane >> 4);
     const int kei_off = G_::KE_OFF + g * ROW_E;
     const int ke_off = G_::KE_OFF + g * ROW_E + ((N == 16) ? 2 * t : (N == 32) ? t : (N == 64) ? (t >> 1) : 0);
-    const int v_off = G_::VM_OFF + t * ROW_M + g * 8;
-    const int ve_off = G_::VE_OFF + t * ROW_E + (16 * g) / N;
-    const int src_lo = 4 * t + (g >> 1), src_hi = 4 * (t + 4) + (g >> 1);
+    int v_off[4], ve_off[4];                                   // bytes [8g, 8g + 8) of rows tok4(t, k)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        v_off[k] = G_::VM_OFF + swz(tok4(t, k), g >> 1) + 8 * (g & 1);
+        ve_off[k] = G_::VE_OFF + tok4(t, k) * ROW_E + (16 * g) / N;
+    }
+    // softmax weights travel from the lanes that computed them (token = lane / 4 and + 8, column pair = lane % 4)
+    const int src_lo = 4 * tok4(t, 0) + (g >> 1), src_hi = 4 * tok4(t, 1) + (g >> 1);
     const uint32_t half_sel = (g & 1) ? 0x7632u : 0x5410u;     // odd columns carry the lo halves
 
     int stage = 0;
@@ -611,11 +604,11 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
         constexpr int VE_WORDS = kTile * ROW_E / 4;      // V exponent bytes of a stage, in words
         // slow path of the check: largest V exponent byte among the tile's live rows; raise the reference to it
         // (plus some headroom, so that small upward steps do not come back here)
-        auto raise_dv = [&](const uint8_t* st, int n_live) {
+        auto raise_dv = [&](const uint8_t* se, int n_live) {
             const int n_bytes = min(n_live, kTile) * ROW_E;
             uint32_t m = 0;
             for (int w = lane; w < VE_WORDS; w += 32) {
-                uint32_t x = *reinterpret_cast<const uint32_t*>(st + G_::VE_OFF + 4 * w);
+                uint32_t x = *reinterpret_cast<const uint32_t*>(se + G_::VE_OFF + 4 * w);
                 const int left = n_bytes - 4 * w;
                 if (left < 4) x = left <= 0 ? 0u : (x & ((1u << (8 * left)) - 1u));
                 m = vmaxu4(m, x);
@@ -657,7 +650,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
         };
 
         // one stage of kTile tokens; FULL = every row of the tile exists
-        auto tile_body = [&](const uint8_t* st, int n_live, auto full_tag) {
+        auto tile_body = [&](const uint8_t* st, const uint8_t* se, int n_live, auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;
             // ---- V exponent bytes against the reference: even and odd bytes in 16-bit lanes, bit 15 = "larger"
             if (FULL) {
@@ -666,13 +659,13 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                 for (int i = 0; i < (VE_WORDS + 31) / 32; ++i) {
                     const int w = lane + 32 * i;
                     if (VE_WORDS % 32 == 0 || w < VE_WORDS) {
-                        const uint32_t x = *reinterpret_cast<const uint32_t*>(st + G_::VE_OFF + 4 * w);
+                        const uint32_t x = *reinterpret_cast<const uint32_t*>(se + G_::VE_OFF + 4 * w);
                         f |= ((x & 0x00FF00FFu) + dv_probe) | (prmt(x, 0u, 0x4341u) + dv_probe);
                     }
                 }
-                if (__any_sync(0xffffffffu, (f & 0x80008000u) != 0u)) raise_dv(st, n_live);
+                if (__any_sync(0xffffffffu, (f & 0x80008000u) != 0u)) raise_dv(se, n_live);
             } else {
-                raise_dv(st, n_live);         // rows past the end may hold anything: masked there
+                raise_dv(se, n_live);         // rows past the end may hold anything: masked there
             }
             // ---- scores ---------------------------------------------------------
             float sc[kMT][NT][2];
@@ -686,8 +679,8 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                 if (MHA) {
                     // ---- single head: lane t feeds bytes [16t, 16t + 16) of tokens g and g + 8; the columns keep the
                     // blocks apart, so all four MMAs go to one accumulator set
-                    const uint4 xa = *reinterpret_cast<const uint4*>(st + G_::KM_OFF + (mt * 16 + g) * ROW_M + 16 * t);
-                    const uint4 xb = *reinterpret_cast<const uint4*>(st + G_::KM_OFF + (mt * 16 + g + 8) * ROW_M + 16 * t);
+                    const uint4 xa = *reinterpret_cast<const uint4*>(st + k_off + mt * 16 * ROW_M);
+                    const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off8 + mt * 16 * ROW_M);
                     int acc[4];
                     mma_u8s8_k32_first(acc, xa.x, xb.x, xa.y, xb.y, qi8[0][0], qi8[0][1], 0, -qbias_h);
                     mma_u8s8_k32(acc, xa.z, xb.z, xa.w, xb.w, qi8[0][4], qi8[0][5]);
@@ -696,8 +689,8 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     // (256 * hi-digit sum + lo-digit sum) * 2^(e_k - 127) * (scale * 2^(qe - 16)) for block t, then the
                     // four blocks of a token are added across the lanes t (an exponent byte of 0 counts as weight 0)
                     constexpr int tb_mask = NBLK - 1;
-                    const uint32_t e0 = st[G_::KE_OFF + (mt * 16 + g) * ROW_E + (t & tb_mask)];
-                    const uint32_t e1 = st[G_::KE_OFF + (mt * 16 + g + 8) * ROW_E + (t & tb_mask)];
+                    const uint32_t e0 = se[G_::KE_OFF + (mt * 16 + g) * ROW_E + (t & tb_mask)];
+                    const uint32_t e1 = se[G_::KE_OFF + (mt * 16 + g + 8) * ROW_E + (t & tb_mask)];
                     float s0 = __int2float_rn(256 * acc[0] + acc[1]) * (__uint_as_float(e0 << 23) * qfac_h);
                     float s1 = __int2float_rn(256 * acc[2] + acc[3]) * (__uint_as_float(e1 << 23) * qfac_h);
                     s0 += __shfl_xor_sync(0xffffffffu, s0, 1);
@@ -706,32 +699,49 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     s1 += __shfl_xor_sync(0xffffffffu, s1, 2);
                     sc[mt][0][0] = s0; sc[mt][0][1] = s1;
                 } else if (KI) {
-                    // ---- integer path: bytes as they are (kind 1) and 16 x low nibble (kind 2), per 16-byte segment
+                    // ---- integer path, several query heads: per 16-byte segment one 32-byte-deep MMA takes the bytes
+                    // as they are (k 0..15) and the words shifted left by four bits (k 16..31; see make_qfrag4i)
                     int acc[NT][NBLK][4];
-                    const uint8_t* pa = st + k_off + mt * 16 * ROW_M;
+                    const uint32_t ka = smem_u32(st) + lm_off + mt * 16 * ROW_M;
+                    constexpr int SEG_PER_BLK = 4 / NBLK;
 #pragma unroll
-                    for (int seg = 0; seg < 4; ++seg) {
-                        const uint32_t wa = *reinterpret_cast<const uint32_t*>(pa + 16 * seg);
-                        const uint32_t wb = *reinterpret_cast<const uint32_t*>(pa + 8 * ROW_M + 16 * seg);
-                        const uint32_t la = (wa << 4) & 0xF0F0F0F0u, lb = (wb << 4) & 0xF0F0F0F0u;    // 16 x low nibble
-                        constexpr int SEG_PER_BLK = 4 / NBLK;
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t w[4];            // rows g, g + 8 of segment 2 half; rows g, g + 8 of segment 2 half + 1
+                        ldmatrix_x4(w[0], w[1], w[2], w[3], half ? (ka ^ 32u) : ka);
 #pragma unroll
-                        for (int nt = 0; nt < NT; ++nt) {
-                            if (seg % SEG_PER_BLK == 0)   // first MMA of a block: the offsets' constant contribution goes in as C
-                                mma_u8s8_first(acc[nt][seg / SEG_PER_BLK], wa, wb, qi8[nt][2 * seg], 0, -qbias[nt][seg / SEG_PER_BLK]);
-                            else
-                                mma_u8s8(acc[nt][seg / SEG_PER_BLK], wa, wb, qi8[nt][2 * seg]);
-                            mma_u8s8(acc[nt][seg / SEG_PER_BLK], la, lb, qi8[nt][2 * seg + 1]);
+                        for (int j = 0; j < 2; ++j) {
+                            const int seg = 2 * half + j, blk = seg / SEG_PER_BLK;
+                            const uint32_t wa = w[2 * j], wb = w[2 * j + 1];
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) {
+                                if (seg % SEG_PER_BLK == 0)   // first MMA of a block: the offsets' constant contribution goes in as C
+                                    mma_u8s8_k32_first(acc[nt][blk], wa, wb, wa << 4, wb << 4, qi8[nt][2 * seg], qi8[nt][2 * seg + 1],
+                                                       0, -qbias[nt][blk]);
+                                else
+                                    mma_u8s8_k32(acc[nt][blk], wa, wb, wa << 4, wb << 4, qi8[nt][2 * seg], qi8[nt][2 * seg + 1]);
+                            }
                         }
                     }
-                    // (256 * hi-digit sum + lo-digit sum) * 2^(e_k - 129) * 2^(qe - 14) * scale, per block
+                    // (256 * hi-digit sum + lo-digit sum) * 2^(e_k - 127) * (scale * 2^(qe - 16)), per block (an exponent
+                    // byte of 0 counts as weight 0)
+                    uint32_t ew0, ew1;            // the exponent bytes of tokens g and g + 8
+                    if (ROW_E == 4) {
+                        ew0 = *reinterpret_cast<const uint32_t*>(se + kei_off + mt * 16 * ROW_E);
+                        ew1 = *reinterpret_cast<const uint32_t*>(se + kei_off + (mt * 16 + 8) * ROW_E);
+                    } else if (ROW_E == 2) {
+                        ew0 = *reinterpret_cast<const uint16_t*>(se + kei_off + mt * 16 * ROW_E);
+                        ew1 = *reinterpret_cast<const uint16_t*>(se + kei_off + (mt * 16 + 8) * ROW_E);
+                    } else {
+                        ew0 = se[kei_off + mt * 16 * ROW_E];
+                        ew1 = se[kei_off + (mt * 16 + 8) * ROW_E];
+                    }
                     float s0[NT], s1[NT];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) s0[nt] = s1[nt] = 0.f;
 #pragma unroll
                     for (int k = 0; k < NBLK; ++k) {
-                        const float w0 = lutf[st[kei_off + mt * 16 * ROW_E + k]];
-                        const float w1 = lutf[st[kei_off + (mt * 16 + 8) * ROW_E + k]];
+                        const float w0 = __uint_as_float(((ew0 >> (8 * k)) & 0xffu) << 23);
+                        const float w1 = __uint_as_float(((ew1 >> (8 * k)) & 0xffu) << 23);
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
                             const float f0 = __int2float_rn(256 * acc[nt][k][0] + acc[nt][k][1]);
@@ -744,13 +754,13 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     for (int nt = 0; nt < NT; ++nt) { sc[mt][nt][0] = s0[nt]; sc[mt][nt][1] = s1[nt]; }
                 } else {
                     const uint4 xa = *reinterpret_cast<const uint4*>(st + k_off + mt * 16 * ROW_M);
-                    const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off + (mt * 16 + 8) * ROW_M);
+                    const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off8 + mt * 16 * ROW_M);
                     const uint32_t wa[4] = {xa.x, xa.y, xa.z, xa.w}, wb[4] = {xb.x, xb.y, xb.z, xb.w};
                     uint2 la[NBK], lb[NBK];
     #pragma unroll
                     for (int k = 0; k < NBK; ++k) {
-                        la[k] = lutk[st[ke_off + mt * 16 * ROW_E + k]];
-                        lb[k] = lutk[st[ke_off + (mt * 16 + 8) * ROW_E + k]];
+                        la[k] = lutk[se[ke_off + mt * 16 * ROW_E + k]];
+                        lb[k] = lutk[se[ke_off + (mt * 16 + 8) * ROW_E + k]];
                     }
                     float acc[NT][2][4];
     #pragma unroll
@@ -833,8 +843,8 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     const float p0 = ex2_approx(sc[mt][0][0] - m_run[0]);
                     const float p1 = ex2_approx(sc[mt][0][1] - m_run[0]);
                     l_run[0] += p0 + p1;
-                    const int ev0 = st[G_::VE_OFF + (mt * 16 + g) * ROW_E + (t & tb_mask)];
-                    const int ev1 = st[G_::VE_OFF + (mt * 16 + g + 8) * ROW_E + (t & tb_mask)];
+                    const int ev0 = se[G_::VE_OFF + (mt * 16 + g) * ROW_E + (t & tb_mask)];
+                    const int ev1 = se[G_::VE_OFF + (mt * 16 + g + 8) * ROW_E + (t & tb_mask)];
                     float w0 = p0 * __int_as_float(max(ev0 + wexp, 0) << 23);
                     float w1 = p1 * __int_as_float(max(ev1 + wexp, 0) << 23);
                     if (!FULL) {       // rows past the end may hold any exponent byte: select, not arithmetic
@@ -845,7 +855,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     const float h0 = __uint_as_float(__float_as_uint(w0) & 0xffffe000u);
                     const float h1 = __uint_as_float(__float_as_uint(w1) & 0xffffe000u);
                     const uint32_t q0 = pack_f16x2_rn(h0, w0 - h0), q1 = pack_f16x2_rn(h1, w1 - h1);
-                    // B fragment for lane (g, t): column g = (block g/2, half g%2); tokens t, t+4 | t+8, t+12
+                    // B fragment for lane (g, t): column g = (block g/2, half g%2); tokens tok4(t, 0), tok4(t, 1) | tok4(t, 2), tok4(t, 3)
                     const uint32_t v0 = __shfl_sync(0xffffffffu, q0, src_lo);
                     const uint32_t v1 = __shfl_sync(0xffffffffu, q0, src_hi);
                     const uint32_t v2 = __shfl_sync(0xffffffffu, q1, src_lo);
@@ -853,7 +863,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     const uint32_t pb0 = prmt(v0, v1, half_sel), pb1 = prmt(v2, v3, half_sel);
                     uint2 vw[4];
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) vw[k] = *reinterpret_cast<const uint2*>(st + v_off + (mt * 16 + 4 * k) * ROW_M);
+                    for (int k = 0; k < 4; ++k) vw[k] = *reinterpret_cast<const uint2*>(st + v_off[k] + mt * 16 * ROW_M);
 #pragma unroll
                     for (int x = 0; x < 4; ++x) {         // byte pair (2x, 2x+1) of the lane's eight bytes
                         const uint32_t wA0 = (x < 2) ? vw[0].x : vw[0].y, wA1 = (x < 2) ? vw[1].x : vw[1].y;
@@ -868,7 +878,7 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     continue;
                 }
                 // softmax weights of this lane's tokens (g and g+8), then the B fragment of P^T for lane (g, t):
-                // column g = (query g/2, half g%2); tokens t, t+4 | t+8, t+12
+                // column g = (query g/2, half g%2); tokens tok4(t, 0), tok4(t, 1) | tok4(t, 2), tok4(t, 3)
                 uint32_t pb[NT][2];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
@@ -880,25 +890,25 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
                     const float h0 = __uint_as_float(__float_as_uint(p0) & 0xffffe000u);
                     const float h1 = __uint_as_float(__float_as_uint(p1) & 0xffffe000u);
                     const uint32_t w0 = pack_f16x2_rn(h0, p0 - h0), w1 = pack_f16x2_rn(h1, p1 - h1);
-                    const uint32_t v0 = __shfl_sync(0xffffffffu, w0, src_lo);   // token t
-                    const uint32_t v1 = __shfl_sync(0xffffffffu, w0, src_hi);   // token t+4
-                    const uint32_t v2 = __shfl_sync(0xffffffffu, w1, src_lo);   // token t+8
-                    const uint32_t v3 = __shfl_sync(0xffffffffu, w1, src_hi);   // token t+12
-                    pb[nt][0] = prmt(v0, v1, half_sel);      // this column's half of tokens (t, t+4)
-                    pb[nt][1] = prmt(v2, v3, half_sel);      // and of tokens (t+8, t+12)
+                    const uint32_t v0 = __shfl_sync(0xffffffffu, w0, src_lo);   // token tok4(t, 0)
+                    const uint32_t v1 = __shfl_sync(0xffffffffu, w0, src_hi);   // token tok4(t, 1)
+                    const uint32_t v2 = __shfl_sync(0xffffffffu, w1, src_lo);   // token tok4(t, 2) = tok4(t, 0) + 8
+                    const uint32_t v3 = __shfl_sync(0xffffffffu, w1, src_hi);   // token tok4(t, 3) = tok4(t, 1) + 8
+                    pb[nt][0] = prmt(v0, v1, half_sel);      // this column's half of the first token pair
+                    pb[nt][1] = prmt(v2, v3, half_sel);      // and of the second
                 }
-                // V pieces: bytes [8g, 8g+8) (slots 16g..16g+15) of tokens t, t+4, t+8, t+12 of this row tile
+                // V pieces: bytes [8g, 8g+8) (slots 16g..16g+15) of tokens tok4(t, 0..3) of this row tile
                 uint2 vw[4];
                 uint2 lv[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    vw[k] = *reinterpret_cast<const uint2*>(st + v_off + (mt * 16 + 4 * k) * ROW_M);
-                    lv[k] = lutv[st[ve_off + (mt * 16 + 4 * k) * ROW_E]];
+                    vw[k] = *reinterpret_cast<const uint2*>(st + v_off[k] + mt * 16 * ROW_M);
+                    lv[k] = lutv[se[ve_off[k] + mt * 16 * ROW_E]];
                 }
                 if (!FULL) {       // rows past the end contribute exactly zero
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        if (mt * 16 + t + 4 * k >= n_live) lv[k] = make_uint2(0u, 0u);
+                        if (mt * 16 + tok4(t, k) >= n_live) lv[k] = make_uint2(0u, 0u);
                 }
                 const uint32_t sA = prmt(lv[0].x, lv[1].x, 0x7610u), cA = prmt(lv[0].y, lv[1].y, 0x7610u);
                 const uint32_t sB = prmt(lv[2].x, lv[3].x, 0x7610u), cB = prmt(lv[2].y, lv[3].y, 0x7610u);
@@ -928,10 +938,11 @@ __global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2) decode_mm
 
         for (int it = 0; it < cr.n_tiles; ++it) {
             if (!mbar_wait_bounded(bar0 + 8 * stage, parity)) { timed_out = true; break; }
-            const uint8_t* st = wsm + stage * G_::STAGE_BYTES;
+            const uint8_t* st = wsm + stage * G_::MANT_STAGE;
+            const uint8_t* se = wse + stage * G_::EXP_STAGE;
             const int n_live = cr.n_tok - it * kTile;        // tokens of this tile that exist (may exceed kTile)
-            if (n_live >= kTile) tile_body(st, n_live, std::true_type{});
-            else tile_body(st, n_live, std::false_type{});
+            if (n_live >= kTile) tile_body(st, se, n_live, std::true_type{});
+            else tile_body(st, se, n_live, std::false_type{});
             if (MHA && ++since_flush == kFlushStages) flush_offsets();
             __syncwarp();
             issue_next(stage);
@@ -1033,10 +1044,16 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     int grid = 0;
     const kvbfp_status st = plan_persistent(a, kTile, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
     if (st != KVBFP_OK) return st;
+    // tensor maps of the two mantissa planes (this device's memory; rows of two tokens, boxes of kTile tokens)
+    CUtensorMap k_map, v_map;
+    const uint64_t n_rows = (uint64_t)a.fmt.batch * a.fmt.n_kv_heads * a.fmt.max_seq;
+    kvbfp_status ms = make_row_map(&k_map, a.k_mant, n_rows / 2, 2 * ROW_M, kTile / 2);
+    if (ms == KVBFP_OK) ms = make_row_map(&v_map, a.v_mant, n_rows / 2, 2 * ROW_M, kTile / 2);
+    if (ms != KVBFP_OK) return ms;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma4<N, NT, MHA><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b, qmeta);
+    decode_mma4<N, NT, MHA><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b, qmeta, k_map, v_map);
     KVBFP_LAUNCH_CHECK("decode_mma4");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;

@@ -1,4 +1,4 @@
-// Inline-PTX helpers shared by the tensor-core decode kernels: mbarrier + 1-D bulk asynchronous
+// Inline-PTX helpers shared by the tensor-core decode kernels: mbarrier, 1-D bulk and tiled 2-D asynchronous
 // copies (one destination thread block each), warp-level MMA, packed 16-bit arithmetic, byte permute, 3-input logic.
 #pragma once
 #include <stdint.h>
@@ -40,6 +40,19 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Tiled 2-D asynchronous copy described by a tensor map (rows of a plane -> one shared-memory tile of this thread
+// block); x counts bytes inside a row and must be a multiple of 16, y counts rows.  Rows outside the tensor arrive as
+// zeros; the barrier always receives the bytes of the whole box.
+__device__ __forceinline__ void tensor_g2s_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+// Four 8 x 16-byte matrices from shared memory: lane i gives the address of row i % 8 of matrix i / 8; lane (g, t)
+// receives bytes 4t..4t+3 of row g of each matrix -- the A-fragment layout of the byte MMAs.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t& d0, uint32_t& d1, uint32_t& d2, uint32_t& d3, uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(d0), "=r"(d1), "=r"(d2), "=r"(d3) : "r"(addr) : "memory");
 }
 __device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {

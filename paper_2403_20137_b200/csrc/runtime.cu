@@ -37,6 +37,40 @@ kvbfp_status sm_count(int* n) {
     return KVBFP_OK;
 }
 
+kvbfp_status make_row_map(CUtensorMap* map, const void* base, uint64_t n_rows, uint32_t row_bytes, uint32_t box_rows) {
+    using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static std::atomic<EncodeFn> encode{nullptr};      // the driver's entry point, asked for once
+    EncodeFn fn = encode.load(std::memory_order_acquire);
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        KVBFP_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q));
+        if (!p || q != cudaDriverEntryPointSuccess) {
+            snprintf(t_err, sizeof t_err, "cuTensorMapEncodeTiled is not available from this driver");
+            return KVBFP_ERR_CUDA;
+        }
+        fn = reinterpret_cast<EncodeFn>(p);
+        encode.store(fn, std::memory_order_release);
+    }
+    if ((row_bytes != 64 && row_bytes != 128) || box_rows < 1 || box_rows > 256 || n_rows < 1 ||
+        n_rows > 0x7fffffffull || !aligned16(base))
+        return KVBFP_ERR_UNSUPPORTED;
+    const cuuint64_t dims[2] = {row_bytes, n_rows};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {row_bytes, box_rows};
+    const cuuint32_t elem[2] = {1, 1};
+    const CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(t_err, sizeof t_err, "cuTensorMapEncodeTiled failed with driver error %d", (int)r);
+        return KVBFP_ERR_CUDA;
+    }
+    return KVBFP_OK;
+}
+
 kvbfp_status status_word(uint32_t** ptr) {
     constexpr int kMaxDev = 64;
     static std::atomic<uint32_t*> cache[kMaxDev];      // per device; two threads asking at once store the same address
