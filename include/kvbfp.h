@@ -273,15 +273,18 @@ kvbfp_status kvbfp_decode_attn_static(const kvbfp_cache* cache, const void* q, k
 
 /*
  * One whole decode step for a caller whose new token lives in HOST memory (Sec. II-A: per step only
- * the new token's q, k, v are computed; the rest is read from the cache): copies k_new, v_new and q
- * to the device, appends the token (kvbfp_append with n_new = 1), runs kvbfp_decode_attn, copies the
+ * the new token's q, k, v are computed; the rest is read from the cache): brings k_new, v_new and q
+ * to the device, appends the token (kvbfp_append with n_new = 1), runs kvbfp_decode_attn, brings the
  * result back and synchronises `stream`, so out_host is valid on return.
- *   k_new_host, v_new_host  host [batch, 1, n_kv_heads, head_dim] of `dt` (pinned memory lets the
- *                           copies run asynchronously)
- *   q_host                  host [batch, n_q_heads, head_dim] of `dt`
- *   out_host                host [batch, n_q_heads, head_dim] f32
+ *   k_new_host, v_new_host  host [batch, 1, n_kv_heads, head_dim] of `dt`, 16-byte aligned
+ *   q_host                  host [batch, n_q_heads, head_dim] of `dt`, 16-byte aligned
+ *   out_host                host [batch, n_q_heads, head_dim] f32, 16-byte aligned
  *   start_pos, seq_lens     device [batch] i32, as in kvbfp_append / kvbfp_decode_attn
  *   staging                 device scratch of at least kvbfp_step_staging_bytes() bytes
+ * How the bytes cross the bus: when all four host buffers are page-locked memory that the current device can
+ * address (cudaHostAlloc / cudaHostRegister; the call asks cudaPointerGetAttributes), the kernels read the new
+ * token and the query from them, and write the result to out_host, in place -- the same bytes cross the bus, without
+ * separate copy commands.  Otherwise (pageable memory) the call falls back to cudaMemcpyAsync through `staging`.
  * All other parameters as in kvbfp_append and kvbfp_decode_attn.
  */
 size_t kvbfp_step_staging_bytes(const kvbfp_format* fmt, int32_t n_q_heads, kvbfp_dtype dt);

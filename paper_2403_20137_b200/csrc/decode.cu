@@ -304,6 +304,27 @@ extern "C" kvbfp_status kvbfp_decode_step_host(const kvbfp_cache* cache, const v
     uint8_t* base = static_cast<uint8_t*>(staging);
     uint8_t *dk = base, *dv = base + up(kv), *dq = base + 2 * up(kv), *dout = base + 2 * up(kv) + up(qb);
     cudaStream_t s = (cudaStream_t)stream;
+    // Page-locked host buffers that this device can address are read and written by the kernels themselves.
+    const void* hp[4] = {k_new_host, v_new_host, q_host, out_host};
+    void* mapped[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool in_place = true;
+    for (int i = 0; i < 4 && in_place; ++i) {
+        cudaPointerAttributes at;
+        const cudaError_t e = cudaPointerGetAttributes(&at, hp[i]);
+        if (e != cudaSuccess) (void)cudaGetLastError();
+        in_place = e == cudaSuccess && at.type == cudaMemoryTypeHost && at.devicePointer != nullptr &&
+                   aligned16(at.devicePointer);
+        mapped[i] = in_place ? at.devicePointer : nullptr;
+    }
+    if (in_place) {
+        kvbfp_status st = kvbfp_append(cache, mapped[0], mapped[1], dt, 1, start_pos, perm_k, perm_v, stream);
+        if (st != KVBFP_OK) return st;
+        st = kvbfp_decode_attn(cache, mapped[2], dt, n_q_heads, seq_lens, max_len_hint, perm_k, inv_perm_v, softmax_scale,
+                               0, static_cast<float*>(mapped[3]), workspace, workspace_bytes, flags, stream);
+        if (st != KVBFP_OK) return st;
+        KVBFP_CUDA(cudaStreamSynchronize(s));
+        return KVBFP_OK;
+    }
     KVBFP_CUDA(cudaMemcpyAsync(dk, k_new_host, kv, cudaMemcpyHostToDevice, s));
     KVBFP_CUDA(cudaMemcpyAsync(dv, v_new_host, kv, cudaMemcpyHostToDevice, s));
     KVBFP_CUDA(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, s));

@@ -7,14 +7,17 @@
 // contiguous range per resident warp; the kernel is persistent (one launch fills the machine once).
 // A warp walks its range as "runs" -- the chunks of one (batch, kv head) that fall into the range --
 // keeping one set of accumulators per run and writing one partial result per run, at the slot of the
-// run's first chunk.  Each warp has a private ring of shared-memory stages filled by 1-D bulk
-// asynchronous copies (lanes 0..3 issue one span each, an mbarrier per stage counts the bytes); the
-// copies run ahead across run boundaries, so a new run starts with its first tiles already on chip.
-// There is no block-wide barrier in the loop; every warp fetches its own tiles.
+// run's first chunk.  Each warp has a private ring of shared-memory stages (an mbarrier per stage counts the
+// bytes): the K and V mantissa tiles of 64 tokens arrive by tiled 2-D asynchronous copies over tensor maps of the
+// two planes (rows of 128 bytes = two tokens, 16-byte pieces swizzled so that every fragment load below is free of
+// bank conflicts), the exponent bytes by 1-D bulk copies; lanes 0..3 issue one piece each.  The copies run ahead
+// across run boundaries, so a new run starts with its first tiles already on chip.  There is no block-wide
+// barrier in the loop; every warp fetches its own tiles.
 //
-// Unpacking is what limits this kernel (integer-pipe instructions, not memory).  A packed byte holds
-// two mantissas in excess-8 code: B = 16*(M_hi+8) + (M_lo+8).  fp16 path (P.V always; scores only for
-// blocks of 16): fp16 has a 10-bit fraction, so the whole byte can be put under the bits of 1024.0 with one byte permute: the element
+// Unpacking is what limits this kernel (instruction issue, not memory).  A packed byte holds
+// two mantissas in excess-8 code: B = 16*(M_hi+8) + (M_lo+8).  fp16 path (P.V with several query heads; scores only
+// for blocks of 16): fp16 has a 10-bit fraction, so the whole byte can be put under the bits of 1024.0 with one byte
+// permute: the element
 // 1024 + B.  A second element with the high nibble masked away and bit 7 set, 1024 + 128 + (M_lo+8),
 // comes from one logic op.  One f16x2 fma per register with the block's power of two removes the
 // common bias 1160 and applies the weight, exactly:
@@ -26,17 +29,10 @@
 //            o_hi = (row1 - row2)/16 once, when the run's partial result is written.
 //
 // Scores for blocks of 32 slots or more use the integer tensor-core path instead (Sec. II-B of the paper:
-// the inner product of two BFP blocks is an integer product plus an exponent addition).  The packed
-// bytes are fed to an unsigned-byte x signed-byte MMA as they are (kind 1) and with the low nibble moved
-// up (kind 2 = 16 x low nibble): two integer ops per packed word and no conversion at all.  The query
-// coefficients c1 = q_hi/16 and c2 = (q_lo - q_hi/16)/16 (both multiply operands that carry a factor 16) of
-// each block are cast to 15-bit fixed point with the block's own exponent and split into two signed
-// byte digits, which sit in two MMA columns; the two 32-bit sums of a (token, block) are recombined
-// exactly, the constant contribution of the offsets (136 per kind-1 byte, 128 per kind-2 byte) was put
-// into the accumulator beforehand, and one fp32 multiply-add applies 2^(e_k + e_q) per (token, block).
+// the inner product of two BFP blocks is an integer product plus an exponent addition); see "integer scores" below.
 //
-// Range of the fp16 path.  fp16 cannot hold 2^e for every exponent byte, so each run first takes the largest
-// exponent byte D of its rows (of V, and of K when the scores use fp16) and uses the weights 2^(e - D + 5): the largest block gets
+// Range of the fp16 path.  fp16 cannot hold 2^e for every exponent byte, so each run keeps a reference exponent
+// byte D of its rows (of V, and of K when the scores use fp16) and uses the weights 2^(e - D + 5): the largest block gets
 // 2^5 (the bias product 1160 * 2^5 still fits fp16), blocks more than 2^29 below the largest one of
 // the run are flushed to zero (their contribution is below 2^-29 of it), and the common factor
 // 2^(D - 134) is applied in fp32 to the partial output (and to fp16 scores).  The weights come from a
@@ -291,9 +287,9 @@ __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_
 
 // One query head per kv head.  With one query the eight MMA columns are free to separate the blocks instead of the
 // queries: column 2*blk + digit holds the coefficient digits of block blk and zeros elsewhere, so ONE accumulator set
-// collects all blocks of a token and lane (g, t) ends up with the two digit sums of (token g, block t).  Lane t feeds
-// bytes [16t, 16t + 16) of a token row: MMA j (0, 1) takes bytes 16t + 8j + (0..3) as k = 4t.., and
-// 16t + 8j + 4 + (0..3) as k = 16 + 4t...  One warp per (batch, kv head).
+// collects all blocks of a token and lane (g, t) ends up with the two digit sums of (token g, block t).  MMA j (0, 1)
+// takes the 16-byte pieces 2j (k = 0..15) and 2j + 1 (k = 16..31) of a token row, lane t bytes 4t..4t+3 of each.  One warp
+// per (batch, kv head).
 __global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta) {
     const int N = a.fmt.block;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gp = lane >> 2, tp = lane & 3;
@@ -310,7 +306,7 @@ __global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta
 #pragma unroll
     for (int wd = 0; wd < 8; ++wd) {
         const int j = wd >> 2, kind = (wd >> 1) & 1, half = wd & 1;
-        const int byte0 = 16 * tp + 8 * j + 4 * half;
+        const int byte0 = 16 * (2 * j + half) + 4 * tp;
         uint32_t reg = 0;
         if (byte0 / (N / 2) == cblk) {
 #pragma unroll
@@ -498,9 +494,9 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
     // per-lane byte offsets inside a stage (mantissa tiles swizzled, see Geo4)
     const int k_off = G_::KM_OFF + swz(g, t);                  // 16 bytes [16t, 16t + 16) of token g,
     const int k_off8 = G_::KM_OFF + swz(g + 8, t);             // of token g + 8
-    // integer scores with several query heads: addresses for the 8 x 16-byte matrix loads.  Lane i names row i % 8 of
-    // matrix i / 8; matrices 0, 1 = rows 0..7 and 8..15 of 16-byte piece 0 (piece 2 with the address bit 5 flipped),
-    // matrices 2, 3 = the same rows of piece 1 (3)
+    // integer scores: addresses for the 8 x 16-byte matrix loads.  Lane i names token row i % 8 of matrix i / 8;
+    // matrices 0, 1 = tokens 0..7 and 8..15 of 16-byte piece 0 (piece j: address ^ (j << 4)), matrices 2, 3 (loads
+    // of four) = the same tokens of piece 1
     const int lm_off = G_::KM_OFF + swz(8 * ((lane >> 3) & 1) + (lane & 7), lane >> 4);
     const int kei_off = G_::KE_OFF + g * ROW_E;
     const int ke_off = G_::KE_OFF + g * ROW_E + ((N == 16) ? 2 * t : (N == 32) ? t : (N == 64) ? (t >> 1) : 0);
@@ -677,22 +673,24 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
                     continue;
                 }
                 if (MHA) {
-                    // ---- single head: lane t feeds bytes [16t, 16t + 16) of tokens g and g + 8; the columns keep the
-                    // blocks apart, so all four MMAs go to one accumulator set
-                    const uint4 xa = *reinterpret_cast<const uint4*>(st + k_off + mt * 16 * ROW_M);
-                    const uint4 xb = *reinterpret_cast<const uint4*>(st + k_off8 + mt * 16 * ROW_M);
+                    // ---- single head: each MMA takes two 16-byte pieces of the token rows (lane t: bytes 4t..4t+3 of each);
+                    // the columns keep the blocks apart, so all four MMAs go to one accumulator set
+                    const uint32_t ka = smem_u32(st) + lm_off + mt * 16 * ROW_M;
+                    uint32_t u[4], v[4];          // tokens g, g + 8 of pieces 0, 1 (u) and 2, 3 (v): bytes 4t..4t+3 of each
+                    ldmatrix_x4(u[0], u[1], u[2], u[3], ka);
+                    ldmatrix_x4(v[0], v[1], v[2], v[3], ka ^ 32u);
                     int acc[4];
-                    mma_u8s8_k32_first(acc, xa.x, xb.x, xa.y, xb.y, qi8[0][0], qi8[0][1], 0, -qbias_h);
-                    mma_u8s8_k32(acc, xa.z, xb.z, xa.w, xb.w, qi8[0][4], qi8[0][5]);
-                    mma_u8s8_k32(acc, xa.x << 4, xb.x << 4, xa.y << 4, xb.y << 4, qi8[0][2], qi8[0][3]);
-                    mma_u8s8_k32(acc, xa.z << 4, xb.z << 4, xa.w << 4, xb.w << 4, qi8[0][6], qi8[0][7]);
+                    mma_u8s8_k32_first(acc, u[0], u[1], u[2], u[3], qi8[0][0], qi8[0][1], 0, 0);
+                    mma_u8s8_k32(acc, v[0], v[1], v[2], v[3], qi8[0][4], qi8[0][5]);
+                    mma_u8s8_k32(acc, u[0] << 4, u[1] << 4, u[2] << 4, u[3] << 4, qi8[0][2], qi8[0][3]);
+                    mma_u8s8_k32(acc, v[0] << 4, v[1] << 4, v[2] << 4, v[3] << 4, qi8[0][6], qi8[0][7]);
                     // (256 * hi-digit sum + lo-digit sum) * 2^(e_k - 127) * (scale * 2^(qe - 16)) for block t, then the
                     // four blocks of a token are added across the lanes t (an exponent byte of 0 counts as weight 0)
                     constexpr int tb_mask = NBLK - 1;
                     const uint32_t e0 = se[G_::KE_OFF + (mt * 16 + g) * ROW_E + (t & tb_mask)];
                     const uint32_t e1 = se[G_::KE_OFF + (mt * 16 + g + 8) * ROW_E + (t & tb_mask)];
-                    float s0 = __int2float_rn(256 * acc[0] + acc[1]) * (__uint_as_float(e0 << 23) * qfac_h);
-                    float s1 = __int2float_rn(256 * acc[2] + acc[3]) * (__uint_as_float(e1 << 23) * qfac_h);
+                    float s0 = __int2float_rn(256 * acc[0] + (acc[1] - qbias_h)) * (__uint_as_float(e0 << 23) * qfac_h);
+                    float s1 = __int2float_rn(256 * acc[2] + (acc[3] - qbias_h)) * (__uint_as_float(e1 << 23) * qfac_h);
                     s0 += __shfl_xor_sync(0xffffffffu, s0, 1);
                     s1 += __shfl_xor_sync(0xffffffffu, s1, 1);
                     s0 += __shfl_xor_sync(0xffffffffu, s0, 2);
@@ -705,21 +703,17 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
                     const uint32_t ka = smem_u32(st) + lm_off + mt * 16 * ROW_M;
                     constexpr int SEG_PER_BLK = 4 / NBLK;
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t w[4];            // rows g, g + 8 of segment 2 half; rows g, g + 8 of segment 2 half + 1
-                        ldmatrix_x4(w[0], w[1], w[2], w[3], half ? (ka ^ 32u) : ka);
+                    for (int seg = 0; seg < 4; ++seg) {
+                        const int blk = seg / SEG_PER_BLK;
+                        uint32_t wa, wb;          // bytes 16 seg + 4t .. + 3 of tokens g and g + 8
+                        ldmatrix_x2(wa, wb, ka ^ (uint32_t)(seg << 4));
 #pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            const int seg = 2 * half + j, blk = seg / SEG_PER_BLK;
-                            const uint32_t wa = w[2 * j], wb = w[2 * j + 1];
-#pragma unroll
-                            for (int nt = 0; nt < NT; ++nt) {
-                                if (seg % SEG_PER_BLK == 0)   // first MMA of a block: the offsets' constant contribution goes in as C
-                                    mma_u8s8_k32_first(acc[nt][blk], wa, wb, wa << 4, wb << 4, qi8[nt][2 * seg], qi8[nt][2 * seg + 1],
-                                                       0, -qbias[nt][blk]);
-                                else
-                                    mma_u8s8_k32(acc[nt][blk], wa, wb, wa << 4, wb << 4, qi8[nt][2 * seg], qi8[nt][2 * seg + 1]);
-                            }
+                        for (int nt = 0; nt < NT; ++nt) {
+                            if (seg % SEG_PER_BLK == 0)   // first MMA of a block starts from zero
+                                mma_u8s8_k32_first(acc[nt][blk], wa, wb, wa << 4, wb << 4, qi8[nt][2 * seg], qi8[nt][2 * seg + 1],
+                                                   0, 0);
+                            else
+                                mma_u8s8_k32(acc[nt][blk], wa, wb, wa << 4, wb << 4, qi8[nt][2 * seg], qi8[nt][2 * seg + 1]);
                         }
                     }
                     // (256 * hi-digit sum + lo-digit sum) * 2^(e_k - 127) * (scale * 2^(qe - 16)), per block (an exponent
@@ -744,8 +738,10 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
                         const float w1 = __uint_as_float(((ew1 >> (8 * k)) & 0xffu) << 23);
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
-                            const float f0 = __int2float_rn(256 * acc[nt][k][0] + acc[nt][k][1]);
-                            const float f1 = __int2float_rn(256 * acc[nt][k][2] + acc[nt][k][3]);
+                            // (the offsets' constant contribution is taken out here: as the accumulator's start value
+                            // it would tie up four registers per block for the whole loop)
+                            const float f0 = __int2float_rn(256 * acc[nt][k][0] + (acc[nt][k][1] - qbias[nt][k]));
+                            const float f1 = __int2float_rn(256 * acc[nt][k][2] + (acc[nt][k][3] - qbias[nt][k]));
                             s0[nt] = fmaf(f0, w0 * qfac[nt][k], s0[nt]);
                             s1[nt] = fmaf(f1, w1 * qfac[nt][k], s1[nt]);
                         }

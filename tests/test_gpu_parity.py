@@ -477,6 +477,37 @@ def test_decode_is_deterministic_and_stream_ordered(oracle, p):
     assert rel_err(host(a).astype(np.float64), ref) <= ATTN_TOL
 
 
+@pytest.mark.parametrize("cfg,pinned", [(2, True), (2, False), (4, True)])
+def test_decode_step_host_equals_device_path(oracle, cfg, pinned):
+    """The step with host buffers (page-locked: read and written in place by the kernels; pageable: copied through
+    the staging buffer) gives bit for bit what append + decode_attn give on device tensors, cache planes included."""
+    w = W.CONFIGS[cfg]
+    Bn, S = 3, 333
+    k, v = W.make_kv(w, n_tokens=S, batch=Bn)
+    q = W.make_q(w, batch=Bn)
+    _, perm, _ = B.calibrate(dev(k.reshape(-1, w.n_kv_heads, 128)), w.n_kv_heads, 128)
+    caches = [B.Cache(Bn, w.n_kv_heads, 128, 336, w.block, w.mant_bits, fill=0) for _ in range(2)]
+    z = dev(torch.zeros(Bn, dtype=torch.int32))
+    sp = dev(torch.full((Bn,), S - 1, dtype=torch.int32))
+    lens = dev(torch.full((Bn,), S, dtype=torch.int32))
+    for c in caches:
+        B.append(c, dev(k[:, :S - 1]), dev(v[:, :S - 1]), z, perm_k=perm)
+    kn, vn = k[:, S - 1:].contiguous(), v[:, S - 1:].contiguous()
+    B.append(caches[0], dev(kn), dev(vn), sp, perm_k=perm)
+    ref = B.decode_attn(caches[0], dev(q), lens, perm_k=perm)
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
+    hk, hv, hq = pin(kn), pin(vn), pin(q.contiguous())
+    hout = pin(torch.zeros(Bn, w.n_q_heads, 128, dtype=torch.float32))
+    staging = torch.empty(B.step_staging_bytes(caches[1].fmt, w.n_q_heads, q.dtype), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(B.decode_workspace_bytes(caches[1].fmt, w.n_q_heads), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                      # twice: the second call rewrites the same row
+        B.decode_step_host(caches[1], hk, hv, hq, sp, lens, hout, staging, ws, perm_k=perm)
+        assert torch.equal(hout, ref.cpu())
+    for name in ("k_mant", "k_exp", "v_mant", "v_exp"):
+        assert torch.equal(getattr(caches[0], name), getattr(caches[1], name)), name
+    assert B.device_status() == 0
+
+
 def test_decode_len_hint_flag(oracle):
     w = W.CONFIGS[2]
     k, v = W.make_kv(w, n_tokens=256)
