@@ -171,153 +171,148 @@ __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t*
 // but 128 for byte 0 of a word) goes into the accumulator beforehand, and one fp32 multiply-add applies
 // 2^(e_k - 127) * scale * log2(e) * 2^(qe - 16) per (token, block) (the factor 2^-2 of the mantissa unit included).
 
-// One warp, one query head: pi(q) -> sq[D]; with q_mant_bits the BFP16 cast of Sec. IV (blocks of N slots, 8-bit
-// mantissas) in place.
-__device__ __forceinline__ void load_query_row(const DecodeArgs& a, int64_t q_row, int hk, bool live, int lane, float* sq) {
-    const int N = a.fmt.block;
-    for (int i = lane; i < D; i += 32) {
-        float v = 0.f;
-        if (live) {
-            const int ch = a.perm_k ? (a.perm_k[hk * D + i] & (D - 1)) : i;
-            const int64_t idx = q_row * D + ch;
-            v = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
-        }
-        sq[i] = v;
-    }
-    __syncwarp();
-    if (a.q_mant_bits) {
-        if (lane < D / N) {
-            float* blk = &sq[lane * N];
-            uint32_t am = 0;
-            for (int j = 0; j < N; ++j) am = max(am, __float_as_uint(blk[j]) & 0x7fffffffu);
-            int e8 = (int)(am >> 23);
-            if (e8 == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e8 = 254; }
-            const int k = 127 - e8 + 6, k1 = k >> 1, k2 = k - k1;
-            const float w = unit_weight(e8, 8);
-            for (int j = 0; j < N; ++j) {
-                const float tv = (blk[j] * pow2i(k1)) * pow2i(k2);
-                blk[j] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * w;
-            }
-        }
-        __syncwarp();
+// With one query head per kv head these coefficients are formed inside the main kernel, by the warp itself at the
+// start of each run and in registers: the query row is 512 bytes, and a launch of its own for it cost more than the
+// arithmetic.  With several heads a small kernel writes them out beforehand (make_qfrag4i).
+
+// What lane L = lane % 16 holds of one query head after query_word(): the digit bytes of packed word L (bytes
+// 4L..4L+3 of a row, slots 8L..8L+7), four per register, for the whole-byte row (a) and the shifted-word row (b), and
+// the factor and the offsets' contribution of the block the word lies in.  Lanes 16..31 do the same for a head of their
+// own (or mirror lanes 0..15).
+struct QWord {
+    uint32_t a_d1, a_d0, b_d1, b_d0;
+    float fac;        // scale * log2(e) * 2^(qe - 16)
+    int bias;         // 136 * sum(C of whole bytes) + 136 * sum(C of shifted bytes), 128 for byte 0 of a word
+};
+// Channels of the eight slots of this lane's word (the permutation of kv head hk, or the identity).
+__device__ __forceinline__ void query_channels(const DecodeArgs& a, int hk, int lane, int (&ch)[8]) {
+    const int L = lane & 15;
+    if (a.perm_k) {
+        const int4 p0 = __ldg(reinterpret_cast<const int4*>(a.perm_k + hk * D + 8 * L));
+        const int4 p1 = __ldg(reinterpret_cast<const int4*>(a.perm_k + hk * D + 8 * L) + 1);
+        ch[0] = p0.x; ch[1] = p0.y; ch[2] = p0.z; ch[3] = p0.w; ch[4] = p1.x; ch[5] = p1.y; ch[6] = p1.z; ch[7] = p1.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) ch[j] = 8 * L + j;
     }
 }
-// One warp, one query head: the coefficient rows of sq[D] as fixed-point integers, sCa[byte] (whole byte) and
-// sCb[byte] (shifted word), and per block meta[2 blk] = scale * log2(e) * 2^(qe - 16) as float bits,
-// meta[2 blk + 1] = the offsets' contribution (meta == nullptr: not written).  Lanes 0..15 own one packed word each
-// (bytes 4 lane .. 4 lane + 3 of the row).
-__device__ __forceinline__ void coefficient_rows(const DecodeArgs& a, const float* sq, int lane, int* sCa, int* sCb, int32_t* meta) {
-    const int N = a.fmt.block, nblk = D / N, wpb = N / 8;       // wpb: 4-byte words per block
-    float ca[4] = {0.f, 0.f, 0.f, 0.f}, cb[4] = {0.f, 0.f, 0.f, 0.f};
-    uint32_t am = 0;
-    if (lane < 16) {
-        float b_next = 0.f;
+// pi(q) of those slots for row q_row of q (!live: a head that does not exist, all zeros).
+__device__ __forceinline__ void query_values(const DecodeArgs& a, int64_t q_row, bool live, const int (&ch)[8], float (&v)[8]) {
 #pragma unroll
-        for (int i = 3; i >= 0; --i) {
-            const int byte = 4 * lane + i;
-            ca[i] = (sq[2 * byte + 1] - b_next) * 0.0625f;
-            cb[i] = (sq[2 * byte] - ca[i]) * 0.0625f;
-            b_next = cb[i];
-            am = max(am, max(__float_as_uint(ca[i]) & 0x7fffffffu, __float_as_uint(cb[i]) & 0x7fffffffu));
+    for (int j = 0; j < 8; ++j) {
+        v[j] = 0.f;
+        if (live) {
+            const int64_t idx = q_row * D + (ch[j] & (D - 1));
+            v[j] = a.q_is_bf16 ? __bfloat162float(static_cast<const __nv_bfloat16*>(a.q)[idx]) : static_cast<const float*>(a.q)[idx];
         }
     }
+}
+// The coefficient rows of one query head from its values v (each half warp may work on a head of its own: nothing
+// crosses the halves); with q_mant_bits first the BFP16 cast of Sec. IV (blocks of N slots, 8-bit mantissas).
+template <int N>
+__device__ __forceinline__ QWord query_word(const DecodeArgs& a, float (&v)[8]) {
+    constexpr int wpb = N / 8;                 // 4-byte words (= lanes) per block
+    if (a.q_mant_bits) {
+        uint32_t am = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) am = max(am, __float_as_uint(v[j]) & 0x7fffffffu);
+#pragma unroll
+        for (int off = wpb >> 1; off; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
+        int e8 = (int)(am >> 23);
+        if (e8 == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e8 = 254; }
+        const int k = 127 - e8 + 6, k1 = k >> 1, k2 = k - k1;
+        const float w = unit_weight(e8, 8);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float tv = (v[j] * pow2i(k1)) * pow2i(k2);
+            v[j] = rintf(fminf(fmaxf(tv, -127.f), 127.f)) * w;
+        }
+    }
+    // byte i of the word: low nibble = slot 2i, high nibble = slot 2i + 1; solved from the last byte down
+    float ca[4], cb[4];
+    uint32_t am = 0;
+    float b_next = 0.f;
+#pragma unroll
+    for (int i = 3; i >= 0; --i) {
+        ca[i] = (v[2 * i + 1] - b_next) * 0.0625f;
+        cb[i] = (v[2 * i] - ca[i]) * 0.0625f;
+        b_next = cb[i];
+        am = max(am, max(__float_as_uint(ca[i]) & 0x7fffffffu, __float_as_uint(cb[i]) & 0x7fffffffu));
+    }
+#pragma unroll
     for (int off = wpb >> 1; off; off >>= 1) am = max(am, __shfl_xor_sync(0xffffffffu, am, off));
     int e = (int)(am >> 23);
     if (e == 255) { raise_flag(a.status, KVBFP_FLAG_NONFINITE); e = 254; }
     const int qe = (am == 0) ? 0 : e - 126;                   // |c| * 2^-qe < 1
     const int sh = 14 - qe, h1 = sh / 2, h2 = sh - h1;        // two exact factors (sh in [-114, 140])
-    int bias = 0;
-    if (lane < 16) {
+    QWord w;
+    w.a_d1 = w.a_d0 = w.b_d1 = w.b_d0 = 0u;
+    w.bias = 0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int Ca = __float2int_rn((ca[i] * pow2i(h1)) * pow2i(h2));
-            const int Cb = __float2int_rn((cb[i] * pow2i(h1)) * pow2i(h2));
-            sCa[4 * lane + i] = Ca;
-            sCb[4 * lane + i] = Cb;
-            bias += 136 * Ca + (i == 0 ? 128 : 136) * Cb;
-        }
+    for (int i = 0; i < 4; ++i) {
+        const int Ca = __float2int_rn((ca[i] * pow2i(h1)) * pow2i(h2));
+        const int Cb = __float2int_rn((cb[i] * pow2i(h1)) * pow2i(h2));
+        w.bias += 136 * Ca + (i == 0 ? 128 : 136) * Cb;
+        const int a1 = (Ca + 128) >> 8, a0 = Ca - 256 * a1;   // C = 256 * d1 + d0, both signed bytes
+        const int b1 = (Cb + 128) >> 8, b0 = Cb - 256 * b1;
+        w.a_d1 |= ((uint32_t)a1 & 0xffu) << (8 * i);  w.a_d0 |= ((uint32_t)a0 & 0xffu) << (8 * i);
+        w.b_d1 |= ((uint32_t)b1 & 0xffu) << (8 * i);  w.b_d0 |= ((uint32_t)b0 & 0xffu) << (8 * i);
     }
-    for (int off = wpb >> 1; off; off >>= 1) bias += __shfl_xor_sync(0xffffffffu, bias, off);
-    if (meta) {
-        if (lane < 16 && lane % wpb == 0) {
-            meta[2 * (lane / wpb)] = __float_as_int(pow2_split(a.scale_log2e, qe - 16));
-            meta[2 * (lane / wpb) + 1] = bias;
-        }
-        if (lane >= 16 && lane < 16 + 4 - nblk) {                 // blocks that do not exist: factor 0, bias 0
-            meta[2 * (nblk + lane - 16)] = 0;
-            meta[2 * (nblk + lane - 16) + 1] = 0;
-        }
-    }
-    __syncwarp();
+#pragma unroll
+    for (int off = wpb >> 1; off; off >>= 1) w.bias += __shfl_xor_sync(0xffffffffu, w.bias, off);
+    w.fac = pow2_split(a.scale_log2e, qe - 16);
+    return w;
 }
 
-// Several query heads per kv head.  One 128-thread block per (batch, kv head, n-tile), one warp per query head of the
-// n-tile.  B fragments of the 32-byte-deep MMAs: word 2 * seg + kind covers the bytes [16 seg, 16 seg + 16) of a row
-// (kind 0: whole bytes, kind 1: shifted words); lane (g, t) holds bytes 4t..4t+3 for column g = (query g/2, digit
-// g%2: 0 = d1, 1 = d0).
+// Several query heads per kv head: one warp per (batch, kv head, n-tile) writes the B fragments of the 32-byte-deep
+// MMAs -- word 2 * seg + kind covers the bytes [16 seg, 16 seg + 16) of a row (kind 0: whole bytes, kind 1: shifted
+// words); lane (g, t) holds bytes 4t..4t+3 for column g = (query g/2, digit g%2: 0 = d1, 1 = d0) -- and, per query
+// head, qmeta[8 q + 2 blk] = factor (float bits), qmeta[8 q + 2 blk + 1] = offsets' contribution.  The two half warps
+// take the query heads (0, 1) of the n-tile, then (2, 3); all loads go out first.
+template <int N>
 __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gp = lane >> 2, tp = lane & 3;
-    const int item = blockIdx.x;
+    constexpr int NBLK = D / N;
+    const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
+    const int item = blockIdx.x * 4 + (threadIdx.x >> 5);
+    if (item >= a.fmt.batch * a.fmt.n_kv_heads * NT) return;
     const int nt = item % NT, hk = (item / NT) % a.fmt.n_kv_heads, b = item / NT / a.fmt.n_kv_heads;
-    const int G = a.n_q_heads / a.fmt.n_kv_heads;
-    __shared__ float sq[4][D];
-    __shared__ int sC[4][2][D / 2];                             // [.][0]: whole-byte row a, [.][1]: shifted-word row b
-    const int qi_w = 4 * nt + warp;                             // this warp's query head within the group
-    const int64_t q_row = (int64_t)b * a.n_q_heads + hk * G + qi_w;
-    load_query_row(a, q_row, hk, qi_w < G, lane, sq[warp]);
-    coefficient_rows(a, sq[warp], lane, sC[warp][0], sC[warp][1], qi_w < G ? qmeta + q_row * 8 : nullptr);
-    __syncthreads();
-    // fragments: word (m, lane) for m = 0..7; thread s writes (m = s / 32, lane) and (m + 4, lane)
-    const int qq = gp >> 1, digit = gp & 1, qi = 4 * nt + qq;
-    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
+    const int Gq = a.n_q_heads / a.fmt.n_kv_heads;
+    int ch[8];
+    float qv[2][8];
+    query_channels(a, hk, lane, ch);
 #pragma unroll
-    for (int mm = 0; mm < 2; ++mm) {
-        const int m = warp + 4 * mm, seg = m >> 1, kind = m & 1;
-        uint32_t reg = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const int C = sC[qq][kind][16 * seg + 4 * tp + e];
-            const int d1 = (C + 128) >> 8, d0 = C - 256 * d1;
-            const int dsel = (qi < G) ? (digit ? d0 : d1) : 0;
-            reg |= ((uint32_t)dsel & 0xffu) << (8 * e);
-        }
-        dst[((m >> 2) * 32 + lane) * 4 + (m & 3)] = reg;
+    for (int pass = 0; pass < 2; ++pass) {
+        const int qi = 4 * nt + 2 * pass + (lane >> 4);
+        query_values(a, (int64_t)b * a.n_q_heads + hk * Gq + (qi < Gq ? qi : 0), qi < Gq, ch, qv[pass]);
     }
-}
-
-// One query head per kv head.  With one query the eight MMA columns are free to separate the blocks instead of the
-// queries: column 2*blk + digit holds the coefficient digits of block blk and zeros elsewhere, so ONE accumulator set
-// collects all blocks of a token and lane (g, t) ends up with the two digit sums of (token g, block t).  MMA j (0, 1)
-// takes the 16-byte pieces 2j (k = 0..15) and 2j + 1 (k = 16..31) of a token row, lane t bytes 4t..4t+3 of each.  One warp
-// per (batch, kv head).
-__global__ void __launch_bounds__(128) make_qfrag4h(DecodeArgs a, int32_t* qmeta) {
-    const int N = a.fmt.block;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, gp = lane >> 2, tp = lane & 3;
-    const int item = blockIdx.x * 4 + warp;                     // (batch, kv head); one query head each
-    __shared__ float sq[4][D];
-    __shared__ int sC[4][2][D / 2];                             // [.][0]: whole-byte row a, [.][1]: shifted-word row b
-    if (item >= a.fmt.batch * a.fmt.n_kv_heads) return;
-    const int hk = item % a.fmt.n_kv_heads;
-    load_query_row(a, item, hk, true, lane, sq[warp]);
-    coefficient_rows(a, sq[warp], lane, sC[warp][0], sC[warp][1], qmeta + (int64_t)item * 8);
-    // fragments: word index 4 j + 2 kind + half (half 0: b0, k = 4t..; half 1: b1, k = 16 + 4t..)
-    const int cblk = gp >> 1, digit = gp & 1;
-    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
+    uint32_t qi8[8];
 #pragma unroll
-    for (int wd = 0; wd < 8; ++wd) {
-        const int j = wd >> 2, kind = (wd >> 1) & 1, half = wd & 1;
-        const int byte0 = 16 * (2 * j + half) + 4 * tp;
-        uint32_t reg = 0;
-        if (byte0 / (N / 2) == cblk) {
+    for (int pass = 0; pass < 2; ++pass) {
+        const QWord w = query_word<N>(a, qv[pass]);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int C = sC[warp][kind][byte0 + i];
-                const int d1 = (C + 128) >> 8, d0 = C - 256 * d1;
-                reg |= ((uint32_t)(digit ? d0 : d1) & 0xffu) << (8 * i);
+        for (int hw = 0; hw < 2; ++hw) {          // the head worked out by half warp hw in this pass
+            const int qq = 2 * pass + hw;
+            const bool mine = (g >> 1) == qq;
+#pragma unroll
+            for (int m = 0; m < 8; ++m) {
+                const int seg = m >> 1, kind = m & 1;
+                const uint32_t d1 = __shfl_sync(0xffffffffu, kind ? w.b_d1 : w.a_d1, 16 * hw + 4 * seg + t);
+                const uint32_t d0 = __shfl_sync(0xffffffffu, kind ? w.b_d0 : w.a_d0, 16 * hw + 4 * seg + t);
+                if (mine) qi8[m] = (g & 1) ? d0 : d1;
+            }
+            const int qi = 4 * nt + qq;
+            if (qi < Gq && (lane & 15) % (N / 8) == 0 && (lane >> 4) == hw) {      // block leaders of that half warp
+                int32_t* meta = qmeta + ((int64_t)b * a.n_q_heads + hk * Gq + qi) * 8;
+                const int k = (lane & 15) / (N / 8);
+                meta[2 * k] = __float_as_int(w.fac);
+                meta[2 * k + 1] = w.bias;
             }
         }
-        dst[((wd >> 2) * 32 + lane) * 4 + (wd & 3)] = reg;
     }
+    static_assert(NBLK >= 1, "");
+    uint32_t* dst = a.qfrag + (int64_t)item * (8 * 32);
+#pragma unroll
+    for (int m = 0; m < 8; ++m) dst[((m >> 2) * 32 + lane) * 4 + (m & 3)] = qi8[m];
 }
 
 // ------------------------------------------------------------------ main kernel
@@ -531,31 +526,49 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
             const uint4* src = reinterpret_cast<const uint4*>(a.qfrag);
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
-                const int qn = 4 * nt + t;
-                const int32_t* meta = qmeta + ((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + (qn < Gq ? qn : 0)) * 8;
                 if (MHA) {
-                    const uint4* s8 = src + ((int64_t)cr.b * Hkv + cr.hk) * (2 * 32);
+                    // B fragments: word 4 j + 2 kind + half covers bytes 16 (2j + half) + 4t .. + 3 (MMA j takes the 16-byte
+                    // pieces 2j and 2j + 1 of a row); column g = (block g / 2, digit g % 2), zeros outside its block
+                    int ch[8];
+                    float qv[8];
+                    query_channels(a, cr.hk, lane, ch);
+                    query_values(a, (int64_t)cr.b * Hkv + cr.hk, true, ch, qv);
+                    const QWord w = query_word<N>(a, qv);
 #pragma unroll
-                    for (int j = 0; j < 2; ++j) {
-                        const uint4 v = __ldg(s8 + j * 32 + lane);
-                        qi8[0][4 * j] = v.x; qi8[0][4 * j + 1] = v.y; qi8[0][4 * j + 2] = v.z; qi8[0][4 * j + 3] = v.w;
+                    for (int wd = 0; wd < 8; ++wd) {
+                        const int j = wd >> 2, kind = (wd >> 1) & 1, half = wd & 1;
+                        const int src_lane = 4 * (2 * j + half) + t;
+                        const uint32_t d1 = __shfl_sync(0xffffffffu, kind ? w.b_d1 : w.a_d1, src_lane);
+                        const uint32_t d0 = __shfl_sync(0xffffffffu, kind ? w.b_d0 : w.a_d0, src_lane);
+                        const bool mine = (16 * (2 * j + half)) / (N / 2) == (g >> 1);
+                        qi8[0][wd] = mine ? ((g & 1) ? d0 : d1) : 0u;
                     }
-                    const int32_t* mh = qmeta + ((int64_t)cr.b * Hkv + cr.hk) * 8;
-                    qfac_h = __int_as_float(mh[2 * t]);
-                    qbias_h = mh[2 * t + 1];
+                    // this lane's block is block t (blocks that do not exist: factor 0, offsets 0)
+                    const int lead = (t < NBLK ? t : 0) * (N / 8);
+                    const float fac = __shfl_sync(0xffffffffu, w.fac, lead);
+                    const int bias = __shfl_sync(0xffffffffu, w.bias, lead);
+                    qfac_h = t < NBLK ? fac : 0.f;
+                    qbias_h = t < NBLK ? bias : 0;
                 } else if (KI) {
+                    // several query heads: fragments and per-block factors come from make_qfrag4i (forming them here, at the
+                    // start of a run, cost this kernel 8 % on long sequences: four heads' worth of dependent loads
+                    // before the first tile can be used)
                     const uint4* s8 = src + (((int64_t)cr.b * Hkv + cr.hk) * NT + nt) * (2 * 32);
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
                         const uint4 v = __ldg(s8 + j * 32 + lane);
                         qi8[nt][4 * j] = v.x; qi8[nt][4 * j + 1] = v.y; qi8[nt][4 * j + 2] = v.z; qi8[nt][4 * j + 3] = v.w;
                     }
+                    const int qn = 4 * nt + t;
+                    const int32_t* meta = qmeta + ((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + (qn < Gq ? qn : 0)) * 8;
 #pragma unroll
                     for (int k = 0; k < NBLK; ++k) {
                         qfac[nt][k] = __int_as_float(meta[2 * k]);
                         qbias[nt][k] = meta[2 * k + 1];
                     }
                 } else {
+                    const int qn = 4 * nt + t;
+                    const int32_t* meta = qmeta + ((int64_t)cr.b * a.n_q_heads + cr.hk * Gq + (qn < Gq ? qn : 0)) * 8;
                     const uint4* s16 = src + (((int64_t)cr.b * Hkv + cr.hk) * NT + nt) * (4 * 32);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
@@ -1032,10 +1045,13 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     int32_t* qmeta = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
                                                (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
-    if (MHA) make_qfrag4h<<<(n_pre + 3) / 4, 128, 0, s>>>(a, qmeta);
-    else if (N >= 32) make_qfrag4i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
-    else make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
-    KVBFP_LAUNCH_CHECK("make_qfrag4");
+    if (N < 32) {
+        make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
+        KVBFP_LAUNCH_CHECK("make_qfrag4");
+    } else if (!MHA) {    // (with one query head per kv head the main kernel forms the query coefficients itself)
+        make_qfrag4i<(N >= 32 ? N : 32)><<<(n_pre + 3) / 4, 128, 0, s>>>(a, NT, qmeta);
+        KVBFP_LAUNCH_CHECK("make_qfrag4i");
+    }
     DecodeArgs b;
     int grid = 0;
     const kvbfp_status st = plan_persistent(a, kTile, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
