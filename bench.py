@@ -294,6 +294,8 @@ def kernel_name(B, w, impl):
         return "decode_mma4"
     if impl != B.DECODE_MMA_BF16 and w.mant_bits == 8 and w.block >= 32:
         return "decode_mma8"
+    if impl != B.DECODE_MMA_BF16 and w.mant_bits == 6 and w.block >= 32 and w.n_q_heads == w.n_kv_heads:
+        return "decode_mma6"
     return "decode_mma"
 
 
@@ -536,7 +538,7 @@ def main():
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f16" if kernel in ("decode_mma4", "decode_mma8") else ("bf16" if kernel == "decode_mma" else "f32"),
+        "dtype": "f16" if kernel in ("decode_mma4", "decode_mma8", "decode_mma6") else ("bf16" if kernel == "decode_mma" else "f32"),
         "data": "synthetic",
         "config": {"workload": workload_name(w), "per_gpu_batch": Bn, "decode_kernel": kernel,
                    "l2": f"inputs larger than L2: {alg / 1e6:.0f} MB of cache read per step vs 126 MB L2",

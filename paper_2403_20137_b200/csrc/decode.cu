@@ -168,10 +168,11 @@ kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype 
     const bool tensor_default = impl != KVBFP_DECODE_SIMT && impl != KVBFP_DECODE_MMA_BF16;
     const bool use_mma4 = tensor_default && f.mant_bits == 4;
     const bool use_mma8 = tensor_default && f.mant_bits == 8 && f.block >= 32;
+    const bool use_mma6 = tensor_default && f.mant_bits == 6 && f.block >= 32 && group == 1;
     int chunk;
     if (chunk_units) {
         chunk = (int)chunk_units * kMinChunk;
-    } else if (use_mma4 || use_mma8) {
+    } else if (use_mma4 || use_mma8 || use_mma6) {
         chunk = kMinChunk;      // the persistent kernel balances by item count: finest items, one partial per range
     } else {
         const int64_t pairs = (int64_t)f.batch * f.n_kv_heads;
@@ -199,6 +200,7 @@ kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype 
     if (impl == KVBFP_DECODE_SIMT) st = launch_decode_simt(a, s);
     else if (use_mma4) st = launch_decode_mma4(a, s, &split);
     else if (use_mma8) st = launch_decode_mma8(a, s, &split);
+    else if (use_mma6) st = launch_decode_mma6(a, s, &split);
     else st = launch_decode_mma(a, s);
     if (st != KVBFP_OK) return st;
     const int n_rows = f.batch * n_q_heads;

@@ -107,6 +107,9 @@ struct Run {
 kvbfp_status launch_decode_mma4(const DecodeArgs& a, cudaStream_t s, Split* split);
 // 8-bit mantissas, blocks of 32 slots or more: integer scores on the stored bytes + fp16 P.V, persistent
 kvbfp_status launch_decode_mma8(const DecodeArgs& a, cudaStream_t s, Split* split);
+// 6-bit mantissas, one query head per kv head, blocks of 32 slots or more: integer scores + fp16 P.V on the stored
+// bytes and their masked copies, persistent
+kvbfp_status launch_decode_mma6(const DecodeArgs& a, cudaStream_t s, Split* split);
 size_t qfrag_bytes(const kvbfp_format& f, int n_q_heads);
 // Events the caller asked to have recorded around the main decode kernel (nullptr = none).
 void profile_events(cudaEvent_t* start, cudaEvent_t* stop);

@@ -394,7 +394,7 @@ def test_decode_empty_and_capacity_edges(oracle, impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("p", [4, 8])
+@pytest.mark.parametrize("p", [4, 6, 8])
 def test_decode_split_invariance(oracle, impl, p):
     """The chunk count must not matter: 1, 2, 7 and 52 chunks agree with each other.  The fp32 kernel
     agrees to 1e-5; the tensor-core kernel carries q and the softmax weights as two bf16 terms
@@ -407,12 +407,16 @@ def test_decode_split_invariance(oracle, impl, p):
         got, ref = run_decode_case(oracle, w, 1, S, [S], 32, p, impl, chunk_tokens=chunk)
         assert rel_err(got, ref) <= ATTN_TOL
         outs.append(got)
+    # The 6-bit single-head kernel feeds the stored V bytes, excess-32 offsets included, to fp16 MMAs whose fp32
+    # accumulation truncates; the offsets are several times the signal, so the bias of a run (about 2^-24 per
+    # accumulation step of what the accumulator holds) shows more, and it changes with the number of steps per run.
+    bound = 1e-5 if impl == B.DECODE_SIMT else (3e-4 if (p == 6 and impl == B.DECODE_MMA) else 1e-4)
     for o in outs[1:]:
-        assert rel_err(o, outs[0]) <= (1e-5 if impl == B.DECODE_SIMT else 1e-4)
+        assert rel_err(o, outs[0]) <= bound
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("p,n", [(4, 16), (4, 32), (4, 128), (8, 32), (8, 64)])
+@pytest.mark.parametrize("p,n", [(4, 16), (4, 32), (4, 128), (8, 32), (8, 64), (6, 32), (6, 128)])
 def test_decode_value_exponents_drift(oracle, impl, p, n):
     """V magnitudes that climb and fall along the sequence, and that jump by 2^60 and up to the top of the
     exponent range for a few tokens: the 4-bit and 8-bit kernels raise the reference exponent of their fp16 V weights
@@ -447,9 +451,11 @@ def test_decode_bfp16_query_and_scale(oracle, impl):
     assert rel_err(got, ref) <= ATTN_TOL
     got, ref = run_decode_case(oracle, w, 1, 300, [300], 32, 8, impl, q_mant_bits=8, scale=0.05)   # 8-bit cache as well
     assert rel_err(got, ref) <= ATTN_TOL
+    got, ref = run_decode_case(oracle, w, 1, 300, [300], 64, 6, impl, q_mant_bits=8, scale=0.05)   # and a 6-bit one
+    assert rel_err(got, ref) <= ATTN_TOL
 
 
-@pytest.mark.parametrize("p", [4, 8])
+@pytest.mark.parametrize("p", [4, 6, 8])
 def test_decode_is_deterministic_and_stream_ordered(oracle, p):
     """Two launches on the same inputs give bit-identical outputs (the work split and the merge order are fixed by
     integer arithmetic, no atomics on the data path), also when the calls are enqueued on a stream of their own
