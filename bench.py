@@ -34,14 +34,16 @@ METRIC = "decode_attn_tokens_per_s"
 UNIT = "tokens/s"
 
 # DRAM traffic of the dominant kernel from one ncu capture (profiles/decode_mma4_b4_s8192_ncu_full.md; the 8-bit
-# kernel: profiles/other_decode_kernels_b4_s8192_ncu_sections.md):
+# kernel: profiles/other_decode_kernels_b4_s8192_ncu_sections.md; the 6-bit one: profiles/decode_mma6_b4_s8192_ncu_sections.md):
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.3093, "block": 32, "mant_bits": 4, "sources_sha256": "b8a7892ca5754edbf44f2cd0313665abe719b15bcbcf55aa9f7cc0db7ef88874"},
-           "decode_mma8": {"bytes_per_unit": 264.3372, "block": 32, "mant_bits": 8, "sources_sha256": "0e0ae313fe6df113eeef12d6dc9031be944ef871e159f7e0f2dd54418cc1c5ce"}}
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.3093, "block": 32, "mant_bits": 4, "sources_sha256": "690fa7de07cde66e9e2e92df7dd47958b5f34ce866ab79a6ce284763ca54955f"},
+           "decode_mma8": {"bytes_per_unit": 264.3797, "block": 32, "mant_bits": 8, "sources_sha256": "f3be562181a11e200ce05ec21744b6e5b8708db23720754468d5d3027d9f9f39"},
+           "decode_mma6": {"bytes_per_unit": 204.1416, "block": 32, "mant_bits": 6, "sources_sha256": "5f3349eaccb5cc834f9f021963d9b3c5ef75b9b6a4e15b69776439a5964fdb47"}}
 KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],
-                  "decode_mma8": ["paper_2403_20137_b200/csrc/decode_mma8.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
+                  "decode_mma8": ["paper_2403_20137_b200/csrc/decode_mma8.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],
+                  "decode_mma6": ["paper_2403_20137_b200/csrc/decode_mma6.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
 
 
 def sources_hash(kernel):
