@@ -386,11 +386,22 @@ def test_decode_group_of_8_and_2(oracle, impl, p, n):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-def test_decode_empty_and_capacity_edges(oracle, impl):
+@pytest.mark.parametrize("p", P_GRID)
+def test_decode_empty_and_capacity_edges(oracle, impl, p):
     w = W.CONFIGS[2]
-    got, ref = run_decode_case(oracle, w, 3, 128, [0, 128, 5], 32, 4, impl, max_seq=128)
+    got, ref = run_decode_case(oracle, w, 3, 128, [0, 128, 5], 32, p, impl, max_seq=128)
     assert not got[0].any() and not ref[0].any()          # empty sequence -> zeros
     assert rel_err(got[1:], ref[1:]) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("p", P_GRID)
+@pytest.mark.parametrize("max_seq,lens", [(16, [16]), (16, [3]), (48, [33]), (80, [80])])
+def test_decode_tiny_caches(oracle, p, max_seq, lens):
+    """Caches smaller than one staged tile (one head, 16 to 80 rows in a plane): the tiled copies of the 4-bit kernel
+    read past the plane's end (zeros arrive) and the kernels must not care."""
+    w = W.CONFIGS[1]
+    got, ref = run_decode_case(oracle, w, 1, lens[0], lens, 32, p, B.DECODE_AUTO, max_seq=max_seq)
+    assert rel_err(got, ref) <= ATTN_TOL
 
 
 @pytest.mark.parametrize("impl", IMPLS)
