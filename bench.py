@@ -38,9 +38,9 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.3093, "block": 32, "mant_bits": 4, "sources_sha256": "690fa7de07cde66e9e2e92df7dd47958b5f34ce866ab79a6ce284763ca54955f"},
-           "decode_mma8": {"bytes_per_unit": 264.3797, "block": 32, "mant_bits": 8, "sources_sha256": "f3be562181a11e200ce05ec21744b6e5b8708db23720754468d5d3027d9f9f39"},
-           "decode_mma6": {"bytes_per_unit": 204.1416, "block": 32, "mant_bits": 6, "sources_sha256": "5f3349eaccb5cc834f9f021963d9b3c5ef75b9b6a4e15b69776439a5964fdb47"}}
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 140.3093, "block": 32, "mant_bits": 4, "sources_sha256": "61dfe7f7fb68a8fdc84bc959de6f6abd1c2f3cccd641c0223756107d502af94a"},
+           "decode_mma8": {"bytes_per_unit": 264.3797, "block": 32, "mant_bits": 8, "sources_sha256": "b046192e7c5e3a98d6a85d578ec3d6b246a370801a397c32a983adf595983b38"},
+           "decode_mma6": {"bytes_per_unit": 204.1416, "block": 32, "mant_bits": 6, "sources_sha256": "39e1112b89fe0d9c252ce3c6a67d3befa7219dd10d60dbf5d765bbe5919d4138"}}
 KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],
                   "decode_mma8": ["paper_2403_20137_b200/csrc/decode_mma8.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],
                   "decode_mma6": ["paper_2403_20137_b200/csrc/decode_mma6.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}

@@ -299,6 +299,16 @@ kvbfp_status kvbfp_decode_step_host(const kvbfp_cache* cache, const void* k_new_
                                     void* stream);
 
 /*
+ * Diagnostic: the bounded barrier wait of the staged decode kernels, on its own.  Launches one warp that waits on a
+ * barrier whose bytes arrive (must succeed) and on one whose bytes nothing ever sends: after `tries` tries of at most
+ * `hint_ns` nanoseconds each (tries <= 1000, hint_ns <= 1 000 000: one second at the most) that wait gives up,
+ * KVBFP_FLAG_WAIT_TIMEOUT is raised in the device status word and the kernel returns normally -- the same thing a
+ * decode kernel does when an on-chip copy does not complete.  Nothing traps and the context stays usable; read the
+ * flag with kvbfp_device_status.  (No counterpart in the paper.)
+ */
+kvbfp_status kvbfp_selftest_wait_timeout(uint32_t tries, uint32_t hint_ns, void* stream);
+
+/*
  * Diagnostics of the work split behind kvbfp_decode_attn (host only: nothing is launched, no device is touched).
  * The persistent kernels lay the sequence pieces ("items") of all (batch, kv head) pairs out pair-major, cut them
  * into one contiguous range per resident warp, and let every range write one partial result per pair it touches;

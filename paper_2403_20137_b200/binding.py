@@ -25,7 +25,8 @@ EXPORTS = ["kvbfp_version", "kvbfp_status_string", "kvbfp_last_cuda_error", "kvb
            "kvbfp_launch_count", "kvbfp_step_staging_bytes", "kvbfp_decode_step_host",
            "kvbfp_profile_decode_events", "kvbfp_static_scratch_bytes", "kvbfp_decode_attn_static",
            "kvbfp_rope_tables", "kvbfp_rope_apply", "kvbfp_decode_attn_rope", "kvbfp_split_plan",
-           "kvbfp_split_range_start", "kvbfp_split_range_of", "kvbfp_split_partial_slot"]
+           "kvbfp_split_range_start", "kvbfp_split_range_of", "kvbfp_split_partial_slot",
+           "kvbfp_selftest_wait_timeout"]
 
 
 class KvbfpError(RuntimeError):
@@ -110,6 +111,7 @@ def lib():
         for name in ("kvbfp_split_range_start", "kvbfp_split_range_of"):
             getattr(L, name).argtypes = [C.c_int32] * 3
             getattr(L, name).restype = C.c_int32
+        L.kvbfp_selftest_wait_timeout.argtypes = [C.c_uint32, C.c_uint32, C.c_void_p]
         L.kvbfp_split_partial_slot.argtypes = [C.c_int32] * 4
         L.kvbfp_split_partial_slot.restype = C.c_int32
         _lib = L
@@ -318,6 +320,11 @@ def profile_decode_events(start=None, stop=None):
     a = None if start is None else C.c_void_p(start.cuda_event)
     b = None if stop is None else C.c_void_p(stop.cuda_event)
     _check(lib().kvbfp_profile_decode_events(a, b))
+
+
+def selftest_wait_timeout(tries=8, hint_ns=1000, stream=None):
+    """kvbfp_selftest_wait_timeout: a bounded barrier wait that must run out; raises FLAG_WAIT_TIMEOUT."""
+    _check(lib().kvbfp_selftest_wait_timeout(tries, hint_ns, _stream(stream)))
 
 
 def static_scratch_bytes():

@@ -18,7 +18,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 // kWaitTries tries the wait gives up and reports failure instead of spinning for ever.
 constexpr uint32_t kWaitHintNs = 1000000u;
 constexpr uint32_t kWaitTries = 2000u;
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_tries(uint32_t bar, uint32_t parity, uint32_t hint_ns, uint32_t tries) {
     uint32_t ok;
     asm volatile(
         "{\n\t"
@@ -34,8 +34,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
         "KVBFP_DONE:\n\t"
         "selp.u32 %0, 1, 0, p;\n\t"
         "}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kWaitHintNs), "r"(kWaitTries) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns), "r"(tries) : "memory");
     return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    return mbar_wait_tries(bar, parity, kWaitHintNs, kWaitTries);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"

@@ -4,6 +4,7 @@
 #include <cstring>
 
 #include "common.cuh"
+#include "ptx.cuh"
 
 namespace kvbfp {
 
@@ -71,6 +72,36 @@ kvbfp_status make_row_map(CUtensorMap* map, const void* base, uint64_t n_rows, u
     return KVBFP_OK;
 }
 
+// Self-test of the bounded barrier wait that every staged kernel relies on: one warp, two barriers.  The first
+// expects 16 bytes that a bulk copy delivers: its wait must succeed.  The second expects 16 bytes that nothing ever
+// sends: its wait must give up after `tries` tries of `hint_ns` each, raise the time-out flag and return -- no trap,
+// nothing left in flight, the context stays usable.
+__device__ __align__(16) uint8_t g_selftest_bytes[16];
+__global__ void __launch_bounds__(32) wait_selftest(uint32_t tries, uint32_t hint_ns, uint32_t* status) {
+    __shared__ __align__(16) uint8_t landing[16];
+    __shared__ __align__(8) uint64_t bars[2];
+    const uint32_t b0 = smem_u32(&bars[0]), b1 = smem_u32(&bars[1]);
+    if (threadIdx.x == 0) {
+        mbar_init(b0, 1);
+        mbar_init(b1, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) {
+        mbar_expect_tx(b0, 16u);
+        bulk_g2s(smem_u32(landing), g_selftest_bytes, 16u, b0);
+        mbar_expect_tx(b1, 16u);                 // bytes that never come
+    }
+    __syncwarp();
+    const bool arrived = mbar_wait_bounded(b0, 0);             // the production bound: the copy lands long before it
+    const bool never = mbar_wait_tries(b1, 0, hint_ns, tries);
+    if (threadIdx.x == 0) {
+        if (!arrived) raise_flag(status, KVBFP_FLAG_NONFINITE);    // (would mean the wait itself is broken)
+        if (!never) raise_flag(status, KVBFP_FLAG_WAIT_TIMEOUT);
+    }
+}
+
 kvbfp_status status_word(uint32_t** ptr) {
     constexpr int kMaxDev = 64;
     static std::atomic<uint32_t*> cache[kMaxDev];      // per device; two threads asking at once store the same address
@@ -115,6 +146,16 @@ kvbfp_status kvbfp_plane_bytes(const kvbfp_format* fmt, size_t* mant_bytes, size
     size_t rows = (size_t)fmt->batch * fmt->n_kv_heads * fmt->max_seq;
     if (mant_bytes) *mant_bytes = rows * kvbfp::row_m_bytes(*fmt);
     if (exp_bytes) *exp_bytes = rows * kvbfp::row_e_bytes(*fmt);
+    return KVBFP_OK;
+}
+
+kvbfp_status kvbfp_selftest_wait_timeout(uint32_t tries, uint32_t hint_ns, void* stream) {
+    if (tries < 1 || tries > 1000 || hint_ns < 1 || hint_ns > 1000000) return KVBFP_ERR_INVALID_ARG;   // at most a second
+    uint32_t* w = nullptr;
+    kvbfp_status st = kvbfp::status_word(&w);
+    if (st != KVBFP_OK) return st;
+    kvbfp::wait_selftest<<<1, 32, 0, (cudaStream_t)stream>>>(tries, hint_ns, w);
+    KVBFP_LAUNCH_CHECK("wait_selftest");
     return KVBFP_OK;
 }
 

@@ -525,6 +525,21 @@ def test_decode_step_host_equals_device_path(oracle, cfg, pinned):
     assert B.device_status() == 0
 
 
+def test_bounded_wait_runs_out_and_context_survives(oracle):
+    """The bounded barrier wait of the staged kernels: a barrier whose bytes never arrive makes the wait give up after
+    its tries, the kernel returns with KVBFP_FLAG_WAIT_TIMEOUT (and only that flag: the barrier whose bytes do arrive
+    was waited for successfully), and the next decode on the same context is correct."""
+    assert B.device_status() == 0
+    B.selftest_wait_timeout(tries=8, hint_ns=1000)
+    assert B.device_status() == B.FLAG_WAIT_TIMEOUT
+    assert B.device_status() == 0                                   # reading clears
+    with pytest.raises(B.KvbfpError):
+        B.selftest_wait_timeout(tries=0)
+    w = W.CONFIGS[1]
+    got, ref = run_decode_case(oracle, w, 1, 256, [256], 16, 4, B.DECODE_AUTO)
+    assert rel_err(got, ref) <= ATTN_TOL
+
+
 def test_decode_len_hint_flag(oracle):
     w = W.CONFIGS[2]
     k, v = W.make_kv(w, n_tokens=256)
