@@ -651,6 +651,14 @@ def test_rope_tables_and_apply(oracle, half_split):
             assert np.allclose(y[r, h], ref_slot, rtol=0, atol=2e-6)
             ref_orig = oracle.rope_apply(x[r, h].astype(np.float64), float(pos[r]), t0, p0, s0)
             assert np.allclose(y[r, h], ref_orig[perm[h]], rtol=0, atol=2e-6)          # commutes with the permutation
+    # runs of consecutive positions far out, with a jump backwards and a repeat in the middle; several row chunks
+    pos2 = np.concatenate([np.arange(31990, 31990 + 45), np.arange(7, 7 + 30), [7, 7, 123456], np.arange(99990, 99990 + 19)]).astype(np.int32)
+    x2 = rng.standard_normal((len(pos2), H, d)).astype(np.float32)
+    y2 = host(B.rope_apply(dev(torch.from_numpy(x2)), dev(torch.from_numpy(pos2)), th, pa, sg)).astype(np.float64)
+    for h in range(H):
+        tp, pp, sp = oracle.rope_permute_tables(perm[h], inv[h], t0, p0, s0)
+        for r in range(len(pos2)):
+            assert np.allclose(y2[r, h], oracle.rope_apply(x2[r, h].astype(np.float64), float(pos2[r]), tp, pp, sp), rtol=0, atol=2e-6)
     # identity tables and bf16 rows
     th1, pa1, sg1 = B.rope_tables(None, None, H, d, 10000.0, half_split)
     xb = torch.from_numpy(x).to(torch.bfloat16)
