@@ -376,6 +376,19 @@ def test_decode_gqa(oracle, impl):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("p,n", [(4, 32), (6, 32), (8, 64), (4, 16)])
+def test_decode_weights_folded_and_vsort(oracle, impl, p, n):
+    """One query head per kv head with the key permutation folded into the weights (perm_k = NULL: the paper's own
+    inference-time setting) and with V-sort (values stored permuted, the output scattered back), ragged lengths."""
+    w = W.CONFIGS[2]
+    lens = [401, 64, 1]
+    got, ref = run_decode_case(oracle, w, 3, 401, lens, n, p, impl, use_perm=False, perm_v=True)
+    assert rel_err(got, ref) <= ATTN_TOL
+    got, ref = run_decode_case(oracle, w, 3, 401, lens, n, p, impl, use_perm=False)
+    assert rel_err(got, ref) <= ATTN_TOL
+
+
+@pytest.mark.parametrize("impl", IMPLS)
 @pytest.mark.parametrize("p,n", [(4, 32), (8, 32), (8, 128), (6, 64)])
 def test_decode_group_of_8_and_2(oracle, impl, p, n):
     import dataclasses
