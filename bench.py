@@ -69,6 +69,12 @@ def workload_name(w):
             f"BFP block{w.block} mant{w.mant_bits}; append 1 token/seq + decode attention")
 
 
+def config_of(w):
+    """The `config` object of both arms: the workload, and how the L2 is kept out of the timing."""
+    return {"workload": workload_name(w),
+            "l2": f"inputs larger than L2: {decode_bytes(w) / 1e6:.0f} MB of cache read per step vs 126 MB L2"}
+
+
 def decode_units(w):
     return w.batch * w.n_kv_heads * w.seq
 
@@ -212,7 +218,7 @@ def run_reference(args, w, rank):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * t_step_full, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(w)},
+        "config": config_of(w),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": st.cores, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -542,10 +548,9 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16" if kernel in ("decode_mma4", "decode_mma8", "decode_mma6") else ("bf16" if kernel == "decode_mma" else "f32"),
         "data": "synthetic",
-        "config": {"workload": workload_name(w), "per_gpu_batch": Bn, "decode_kernel": kernel,
-                   "l2": f"inputs larger than L2: {alg / 1e6:.0f} MB of cache read per step vs 126 MB L2",
-                   "device_status_flags": flags, "e2e_matches_device_path": e2e_ok,
-                   "tokens_per_s_if_32_layers": value / 32.0},
+        "config": config_of(w),
+        "details": {"per_gpu_batch": Bn, "decode_kernel": kernel, "device_status_flags": flags,
+                    "e2e_matches_device_path": e2e_ok, "tokens_per_s_if_32_layers": value / 32.0},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": (ms_e2e / args.steps) if n_e2e else None},
