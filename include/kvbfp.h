@@ -74,10 +74,11 @@ enum {
     KVBFP_DECODE_SIMT = 1,     /* fp32 FMA on the plain ALUs, one query head at a time                */
     KVBFP_DECODE_MMA = 2,      /* same as AUTO: grouped queries as the N operand of warp-level MMAs   */
     KVBFP_DECODE_MMA_BF16 = 3  /* the generic bf16 tensor-core kernel (all mantissa widths).  AUTO uses the
-                                  integer-score kernels for 4 bits and for 8 bits with blocks of 32 or more,
-                                  and this one otherwise (6 bits; 8 bits with blocks of 16).  Its conversion
-                                  leaves the bf16 range for cache values of magnitude 2^120 and above; the
-                                  other kernels have no such limit. */
+                                  integer-score kernels for 4 bits, for 8 bits with blocks of 32 or more and for
+                                  6 bits with blocks of 32 or more and one query head per kv head, and this one
+                                  otherwise (6 bits with grouped query heads or blocks of 16; 8 bits with blocks
+                                  of 16).  Its conversion leaves the bf16 range for cache values of magnitude
+                                  2^120 and above; the other kernels have no such limit. */
 };
 /* Optional, or-ed into `flags`: tokens per sequence chunk (a multiple of 128; 0 = chosen by the
  * library from the batch size and the sequence bound). */
