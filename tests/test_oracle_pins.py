@@ -593,3 +593,67 @@ def test_workload_recipe():
     assert k.dtype.is_floating_point and k.shape == (1, 64, 32, 128) and bool((k == k2).all())
     sd = k.float().std(dim=(0, 1))
     assert float(sd[0, ch[0, 0]]) > 3.0 and abs(float(v.float().std()) - 1.0) < 0.05
+
+
+# ------------------------------------------------------------------------------- values the paper prints
+def _golden(name):
+    import os
+    out = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            if ":" in line:
+                k, v = line.split(":", 1)
+                out[k.strip()] = [float(x) for x in v.split()]
+            else:
+                parts = line.split()
+                out[parts[0]] = [float(x) for x in parts[1:]]
+    return out
+
+
+def test_rope_tables_match_the_vectors_the_paper_prints(oracle):
+    """Sec. III and its footnote print the frequency, partner-index and sign vectors of the rotary embedding; the
+    oracle's tables for a head of 8 channels must be exactly those (tests/golden/rope_order_sec3.txt)."""
+    g = _golden("rope_order_sec3.txt")
+    d, base = 8, g["base"][0]
+    theta, partner, sign = oracle.rope_tables(d, base, False)
+    want_theta = np.array([base ** (-2.0 * (i - 1) / d) for i in g["theta_index_interleaved"]])
+    assert np.allclose(theta, want_theta, rtol=1e-15, atol=0)
+    assert np.array_equal(partner + 1, np.array(g["partner_interleaved"], dtype=np.int32))
+    assert np.array_equal(sign, np.array(g["sign_interleaved"]))
+    theta_h, partner_h, sign_h = oracle.rope_tables(d, base, True)
+    want_h = np.array([base ** (-2.0 * (i - 1) / d) for i in g["theta_index_half_split"]])
+    assert np.allclose(theta_h, want_h, rtol=1e-15, atol=0)
+    # partners share a frequency and carry opposite signs in both layouts
+    for th, pa, sg in ((theta, partner, sign), (theta_h, partner_h, sign_h)):
+        assert np.array_equal(th[pa], th) and np.array_equal(sg[pa], -sg) and np.array_equal(pa[pa], np.arange(d))
+
+
+def test_formats_match_the_ranges_the_paper_prints(oracle):
+    """Sec. II-B prints the mantissa range and the two formats in use; the cast must reach both ends of the range and
+    never leave it, and a block as large as the head makes K-sort a no-op (Table I, block 128)
+    (tests/golden/bfp_formats_sec2b.txt)."""
+    g = _golden("bfp_formats_sec2b.txt")
+    rng = np.random.default_rng(5)
+    for name in ("BFP12", "BFP16"):
+        p, b, lo, hi = (int(x) for x in g[name])
+        assert b == 8 and lo == -(2 ** (p - 1) - 1) and hi == 2 ** (p - 1) - 1
+        scale = np.exp2(float(rng.integers(-20, 20)))
+        x = rng.uniform(-0.9, 0.9, 32) * scale
+        x[3], x[7] = 1.999 * scale, -1.999 * scale          # both ends round past the range and are clamped to it
+        e8, M = oracle.bfp_cast_block(x, p)
+        assert M.min() == lo and M.max() == hi and 0 < e8 < 255
+        assert np.isclose(p + b / 32.0, {4: 4.25, 8: 8.25}[p])
+    assert g["table1_block128_ksort_equals_unsorted"] == [1.0]
+    d = 128
+    k = (rng.standard_normal((1, 40, 1, d)) * np.where(rng.random(d) < 0.05, 20.0, 1.0)).astype(np.float32)
+    _, perm, _ = oracle.calibrate(k.reshape(-1, 1, d), "f32", 1, d)
+    plain, sortd = oracle.Cache(1, 1, d, 48, 128, 4), oracle.Cache(1, 1, d, 48, 128, 4)
+    z = np.zeros(1, np.int32)
+    oracle.append(plain, k, None, "f32", z)
+    oracle.append(sortd, k, None, "f32", z, perm_k=perm)
+    a = oracle.dequant(plain, "k", 0, 0, 0, 40)
+    b_ = oracle.dequant(sortd, "k", 0, 0, 0, 40, perm=perm)
+    assert np.array_equal(a, b_)
