@@ -553,6 +553,26 @@ def test_bounded_wait_runs_out_and_context_survives(oracle):
     assert rel_err(got, ref) <= ATTN_TOL
 
 
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("p", P_GRID)
+def test_decode_zero_query_is_the_mean_of_values(oracle, impl, p):
+    """A query of zeros scores every token alike: the output is the plain mean of the cached values (the fixed-point
+    query coefficients of the integer kernels are all zero then, with exponent zero)."""
+    w = W.CONFIGS[2]
+    Bn, S = 2, 200
+    k, v = W.make_kv(w, n_tokens=S, batch=Bn)
+    q = torch.zeros(Bn, w.n_q_heads, 128, dtype=W.torch_dtype(w.dtype))
+    oc = oracle_cache(oracle, k, v, w.dtype, 32, p, 208)
+    ref = oracle.decode_attn(oc, W.to_oracle(q), w.dtype, w.n_q_heads, [S, 77])
+    gc = B.Cache(Bn, w.n_kv_heads, 128, 208, 32, p, fill=0xFF)
+    B.append(gc, dev(k), dev(v), dev(torch.zeros(Bn, dtype=torch.int32)))
+    out = host(B.decode_attn(gc, dev(q), dev(torch.tensor([S, 77], dtype=torch.int32)), impl=impl)).astype(np.float64)
+    assert B.device_status() == 0
+    assert rel_err(out, ref) <= ATTN_TOL
+    vd = np.stack([oracle.dequant(oc, "v", 1, h, 0, 77) for h in range(w.n_kv_heads)])       # [H, 77, d]
+    assert rel_err(out[1], vd.mean(axis=1)) <= ATTN_TOL
+
+
 def test_decode_len_hint_flag(oracle):
     w = W.CONFIGS[2]
     k, v = W.make_kv(w, n_tokens=256)
