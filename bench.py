@@ -438,7 +438,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the set-up timings, the quality report and the further "
                     "configurations (GQA layer, mantissa sweep)")
-    ap.add_argument("--sweep5", action="store_true", help="add the prefill/append and calibration sweep (8 KV heads, 65536 new\n                    tokens, blocks 16/32/64 x mantissas 4/6/8, calibration over 2^20 tokens) to the extras")
+    ap.add_argument("--sweep5", action="store_true", help="(kept for old command lines: the sweep is part of the default run)")
+    ap.add_argument("--no-sweep5", action="store_true", help="skip the prefill/append and calibration sweep (8 KV heads, 65536 "
+                    "new tokens, blocks 16/32/64 x mantissas 4/6/8, calibration over 2^20 tokens, read-back paths) in the extras")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
     over = {k: v for k, v in (("batch", args.batch), ("seq", args.seq), ("mant_bits", args.mant_bits),
@@ -480,8 +482,6 @@ def main():
     if not args.no_extras:
         extras.update(rig.setup_timings())
     rig.free_setup()
-    if args.sweep5 and rank == 0:
-        extras["config5"] = sweep_config5(B, dev)
 
     # ---- device-resident timing: the step metric, then the main kernel's own duration ---------------
     sampler = ClockSampler(local_rank)
@@ -528,6 +528,8 @@ def main():
         extras["config4"] = side_config(B, W.CONFIGS[4], dev, impl, 300, 10, local_rank, barrier)
         extras["mant_sweep"] = {f"p{p}": side_config(B, dataclasses.replace(w, mant_bits=p), dev, impl, 300, 10,
                                                      local_rank, barrier) for p in (6, 8)}
+    if not args.no_extras and world == 1 and not args.no_sweep5 and not over and args.config == 3:
+        extras["config5"] = sweep_config5(B, dev)
     if not args.no_extras and world == 1:
         from paper_2403_20137_b200 import quality as Q
         nq = max(16, min(2048, S // 16 * 16))
