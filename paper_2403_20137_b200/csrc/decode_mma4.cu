@@ -54,8 +54,12 @@ constexpr int kWarps = 4;
 constexpr int kMT = 4;                  // 16-token MMA row tiles per stage
 constexpr int kTile = 16 * kMT;         // tokens per stage
 constexpr int kStages = 2;
-constexpr int kMinCtas = 3;             // resident thread blocks per SM with one 8-column tile; two tiles (groups of 5 to
-                                        // 8 heads) run two blocks per SM: with three they spill, and measured 9 % slower
+constexpr int kMinCtas = 3;             // resident thread blocks per SM with several query heads in one 8-column tile; two
+                                        // tiles (groups of 5 to 8 heads) run two blocks per SM: with three they spill, and
+                                        // measured 9 % slower
+constexpr int kMinCtasSingle = 2;       // one query head per kv head: two blocks (8 warps) per SM with up to 255 registers
+                                        // measured 4 % faster than three (0.91 against 0.87 of the copy bandwidth on the
+                                        // same box); grouped heads the other way round (0.73 against 0.76)
 constexpr int D = kHeadDim;
 constexpr int ROW_M = D / 2;            // 64 bytes of mantissas per token row
 constexpr int kTopShift = 5;            // weight of the run's largest block is 2^kTopShift
@@ -386,7 +390,7 @@ __device__ __forceinline__ int warp_max_byte(const uint8_t* p, int bytes, int la
 // MHA: one query head per kv head and blocks of 32 slots or more -- the MMA columns separate the blocks of a row
 // instead of the query heads (see make_qfrag4h), in the scores and in P.V.
 template <int N, int NT, bool MHA>
-__global__ void __launch_bounds__(kWarps * 32, NT == 1 ? kMinCtas : 2)
+__global__ void __launch_bounds__(kWarps * 32, MHA ? kMinCtasSingle : (NT == 1 ? kMinCtas : 2))
 decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_constant__ CUtensorMap k_map,
             const __grid_constant__ CUtensorMap v_map) {
     using G_ = Geo4<N>;
