@@ -177,6 +177,44 @@ def test_append_ragged_positions_and_flags(oracle):
     assert B.device_status() & B.FLAG_NONFINITE
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("p", P_GRID)
+def test_append_runs_ragged_tiles_and_nonfinite(oracle, dtype, p):
+    """Runs of tokens (16 and more per sequence: the kernel that stages rows in shared memory) whose length leaves a
+    tile with one row, with three rows and with a full tile less one; two sequences at different positions, both
+    sides permuted.  Then an Inf and a NaN in two rows: flagged, every row without them unchanged."""
+    rng = np.random.default_rng(21)
+    H = 3
+    perm_k = np.stack([rng.permutation(128) for _ in range(H)]).astype(np.int32)
+    perm_v = np.stack([rng.permutation(128) for _ in range(H)]).astype(np.int32)
+    base_k, base_v = adversarial_rows(dtype, seed=22), adversarial_rows(dtype, seed=23)      # [1, 96, 2, 128]
+    for T in (16, 17, 19, 47, 96):
+        k = base_k.repeat(2, 1, 2, 1)[:, :T, :H].contiguous()
+        v = base_v.repeat(2, 1, 2, 1)[:, :T, :H].contiguous()
+        k[1] = k[1].flip(0)
+        start = [5, 0]
+        gc = B.Cache(2, H, 128, 112, 32, p, fill=0xC3)
+        B.append(gc, dev(k), dev(v), dev(torch.tensor(start, dtype=torch.int32)), dev(torch.from_numpy(perm_k)),
+                 dev(torch.from_numpy(perm_v)))
+        assert B.device_status() == 0
+        oc = oracle_cache(oracle, k, v, dtype, 32, p, 112, start=start, perm_k=perm_k, perm_v=perm_v)
+        assert_planes_equal(gc, oc, [T, T], start=start)
+        assert bool((gc.k_mant[0, :, :5] == 0xC3).all()) and bool((gc.v_exp[1, :, T:] == 0xC3).all())
+        assert bool((gc.v_mant[0, :, 5 + T:] == 0xC3).all()) and bool((gc.k_exp[0, :, :5] == 0xC3).all())
+    bad = k.clone()
+    bad[0, 18, 1, 9] = float("inf")
+    bad[1, 95, 2, 127] = float("nan")
+    gb = B.Cache(2, H, 128, 112, 32, p, fill=0xC3)
+    B.append(gb, dev(bad), dev(v), dev(torch.tensor(start, dtype=torch.int32)), dev(torch.from_numpy(perm_k)),
+             dev(torch.from_numpy(perm_v)))
+    assert B.device_status() == B.FLAG_NONFINITE
+    same = torch.ones(2, H, 112, dtype=torch.bool)
+    same[0, 1, 5 + 18] = False
+    same[1, 2, 95] = False
+    assert bool((gb.k_mant.cpu()[same] == gc.k_mant.cpu()[same]).all()) and bool((gb.k_exp.cpu()[same] == gc.k_exp.cpu()[same]).all())
+    assert bool((gb.v_mant == gc.v_mant).all())
+
+
 # ------------------------------------------------------------------------------- calibrate
 @pytest.mark.parametrize("cfg,T", [(1, 256), (2, 1000), (4, 777)])
 def test_calibrate_matches_oracle(oracle, cfg, T):
