@@ -410,7 +410,8 @@ kvbfp_status launch_rows(const AppendArgs& a, cudaStream_t s) {
     int n_sm = 0;
     const kvbfp_status st = sm_count(&n_sm);
     if (st != KVBFP_OK) return st;
-    // one resident wave: as many thread blocks as the device holds at once, split over the sides that have rows
+    // thread blocks over the sides that have rows: one resident wave where blocks of one (sequence, head) fill at
+    // least 15/16 of it, else about eight waves of shorter blocks, which even out; no block shorter than 16 tiles
     static std::atomic<int> per_sm{0};              // (two host threads asking at once store the same number)
     int bps = per_sm.load(std::memory_order_relaxed);
     if (bps == 0) {
@@ -419,12 +420,16 @@ kvbfp_status launch_rows(const AppendArgs& a, cudaStream_t s) {
         per_sm.store(bps, std::memory_order_relaxed);
     }
     const int sides = (a.src[0] ? 1 : 0) + (a.src[1] ? 1 : 0);
-    const int64_t per_chunk = (int64_t)a.n_heads * a.batch;
-    int64_t chunks = (int64_t)n_sm * bps / sides / per_chunk;          // rounded down: no thread block waits for a second wave
-    if (chunks > tiles) chunks = tiles;
+    const int64_t per_chunk = (int64_t)a.n_heads * a.batch * sides;
+    const int64_t resident = (int64_t)n_sm * bps;
+    int64_t chunks = resident / per_chunk;                              // one wave, if blocks of equal length fill it
+    if (chunks * per_chunk * 16 < resident * 15 || chunks > tiles / 16) {
+        chunks = (8 * resident + per_chunk - 1) / per_chunk;
+        if (chunks > tiles / 16) chunks = tiles / 16;
+    }
     if (chunks < 1) chunks = 1;
     if (per_chunk * chunks > 0x7fffffffLL) return KVBFP_ERR_UNSUPPORTED;
-    dim3 grid((unsigned)(per_chunk * chunks), 2, 1);
+    dim3 grid((unsigned)(per_chunk / sides * chunks), 2, 1);
     append_rows<P, N, T><<<grid, kThreads, 0, s>>>(a, (int)chunks);
     KVBFP_LAUNCH_CHECK("append_rows");
     return KVBFP_OK;
