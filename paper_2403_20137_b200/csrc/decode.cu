@@ -28,47 +28,54 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
     const int nc = (len + item_tokens - 1) / item_tokens;        // items that hold tokens
     const float* base = partials + (int64_t)row * n_chunks * kPartStride;
     const int first = (b * (n_q_heads / group) + hq / group) * items_per_pair;   // first item of the pair
+    // The partials of the row: with n_warps == 0 one per item; else one per range that holds items of the pair --
+    // the ranges are consecutive, and the k-th of them starts inside the pair at the first item of range w0 + k
+    // (the first one at item 0), so every lane finds its own partial without walking the others.
+    int w0 = 0, n_part = nc;
+    if (n_warps > 0 && nc > 0) {
+        w0 = range_of(first, range_items, range_extra);
+        n_part = range_of(first + nc - 1, range_items, range_extra) - w0 + 1;
+    }
     float m = -INFINITY, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int i = 0; i < nc;) {
-        // up to eight partials at a time: first their slots (integer arithmetic only), then all loads together
-        int slot[8];
-        int cnt = 0;
+    for (int k0 = 0; k0 < n_part; k0 += 32) {
+        // a lane per partial: its slot, maximum and sum; then the weights of all 32 against the common maximum
+        const int k = k0 + lane;
+        const bool have = k < n_part;
+        int item = k;
+        if (n_warps > 0) item = max(range_start(w0 + (have ? k : 0), range_items, range_extra) - first, 0);
+        const int slot = have ? partial_slot(item, item_tokens, chunk, n_chunks) : 0;
+        const float* pk = base + (int64_t)slot * kPartStride;
+        const float mk = have ? pk[D] : -INFINITY;
+        const float lk = have ? pk[D + 1] : 0.f;
+        float mn = mk;
 #pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            slot[k] = i;
-            if (i < nc) {
-                ++cnt;
-                if (n_warps == 0) {
-                    ++i;
-                } else {                             // next partial of the pair: where the next range starts
-                    const int w = range_of(first + i, range_items, range_extra);    // range that holds this item
-                    i = range_start(w + 1, range_items, range_extra) - first;
-                }
+        for (int off = 16; off; off >>= 1) mn = fmaxf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
+        mn = fmaxf(mn, m);
+        const float a1 = (m == -INFINITY) ? 0.f : exp2f(m - mn);
+        const float ak = (mk == -INFINITY) ? 0.f : exp2f(mk - mn);
+        float ls = ak * lk;
+#pragma unroll
+        for (int off = 16; off; off >>= 1) ls += __shfl_xor_sync(0xffffffffu, ls, off);
+        acc.x *= a1; acc.y *= a1; acc.z *= a1; acc.w *= a1;
+        l = l * a1 + ls;
+        m = mn;
+        // the vectors, eight loads at a time: lane j's slot and weight go round, every lane adds its four channels
+        const int cnt = min(32, n_part - k0);
+        for (int j0 = 0; j0 < cnt; j0 += 8) {
+            float4 oi[8];
+            float aj[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int sj = __shfl_sync(0xffffffffu, slot, (j0 + u) & 31);
+                aj[u] = __shfl_sync(0xffffffffu, ak, (j0 + u) & 31);       // 0 for lanes without a partial
+                oi[u] = *reinterpret_cast<const float4*>(base + (int64_t)sj * kPartStride + lane * 4);
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                acc.x += aj[u] * oi[u].x; acc.y += aj[u] * oi[u].y; acc.z += aj[u] * oi[u].z; acc.w += aj[u] * oi[u].w;
             }
         }
-        float mi[8], li[8];
-        float4 oi[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const float* p = base + (int64_t)(k < cnt ? partial_slot(slot[k], item_tokens, chunk, n_chunks) : 0) * kPartStride;
-            mi[k] = (k < cnt) ? p[D] : -INFINITY;
-            li[k] = (k < cnt) ? p[D + 1] : 0.f;
-            oi[k] = (k < cnt) ? *reinterpret_cast<const float4*>(p + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        float mn = m;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) mn = fmaxf(mn, mi[k]);
-        const float a1 = (m == -INFINITY) ? 0.f : exp2f(m - mn);
-        acc.x *= a1; acc.y *= a1; acc.z *= a1; acc.w *= a1;
-        l *= a1;
-#pragma unroll
-        for (int k = 0; k < 8; ++k) {
-            const float a2 = (mi[k] == -INFINITY) ? 0.f : exp2f(mi[k] - mn);
-            acc.x += a2 * oi[k].x; acc.y += a2 * oi[k].y; acc.z += a2 * oi[k].z; acc.w += a2 * oi[k].w;
-            l += a2 * li[k];
-        }
-        m = mn;
     }
     const float inv = (l > 0.f) ? 1.f / l : 0.f;
     float* dst = out + (int64_t)row * D;
