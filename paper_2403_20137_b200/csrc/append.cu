@@ -62,6 +62,8 @@ __global__ void __launch_bounds__(kThreads) append_quant_pack(AppendArgs a) {
     constexpr float MAGIC = 12582912.f + (float)EXC;            // 1.5 * 2^23 + 2^(p-1)
     constexpr uint32_t MAGIC_BITS = 0x4B400000u;                // bits of 1.5 * 2^23: sum bits - this = field
 
+    pdl_wait();
+    pdl_trigger();
     const int which = blockIdx.y;
     const T* src = static_cast<const T*>(a.src[which]);
     if (!src) return;
@@ -203,6 +205,8 @@ __global__ void __launch_bounds__(kThreads) append_rows(AppendArgs a, int chunks
     constexpr int EXC = 1 << (P - 1), QMAX = EXC - 1;
     __shared__ __align__(128) uint8_t ring[kWarps * kRing * STAGE_BYTES];
 
+    pdl_wait();
+    pdl_trigger();
     const int which = blockIdx.y;
     const T* src = static_cast<const T*>(which ? a.src[1] : a.src[0]);
     if (!src) return;
@@ -430,7 +434,7 @@ kvbfp_status launch_rows(const AppendArgs& a, cudaStream_t s) {
     if (chunks < 1) chunks = 1;
     if (per_chunk * chunks > 0x7fffffffLL) return KVBFP_ERR_UNSUPPORTED;
     dim3 grid((unsigned)(per_chunk / sides * chunks), 2, 1);
-    append_rows<P, N, T><<<grid, kThreads, 0, s>>>(a, (int)chunks);
+    (void)launch_pdl(append_rows<P, N, T>, grid, dim3(kThreads), 0, s, a, (int)chunks);
     KVBFP_LAUNCH_CHECK("append_rows");
     return KVBFP_OK;
 }
@@ -449,7 +453,7 @@ kvbfp_status launch(const AppendArgs& a, int64_t n_rows, cudaStream_t s) {
     if (hs > a.n_heads) hs = a.n_heads;
     if (hs < 1) hs = 1;
     dim3 grid(gx, 2, hs);
-    append_quant_pack<P, N, T><<<grid, kThreads, 0, s>>>(a);
+    (void)launch_pdl(append_quant_pack<P, N, T>, grid, dim3(kThreads), 0, s, a);
     KVBFP_LAUNCH_CHECK("append_quant_pack");
     return KVBFP_OK;
 }

@@ -57,6 +57,32 @@ inline size_t row_e_bytes(const kvbfp_format& f) { return (size_t)(f.head_dim / 
 
 // ---- device side -----------------------------------------------------------
 
+// ---- launches that overlap with the kernel before them -----------------------
+//
+// The kernels of a decode step (cache write, query coefficients, attention, merge) are launched with programmatic
+// stream serialization: the next kernel's thread blocks may become resident and run their set-up while the kernel
+// before it is still running.  Every such kernel calls pdl_wait() before its first access to global memory (it
+// returns once the kernel before it has completed and its writes are visible; at once if the launch had no such
+// predecessor) and pdl_trigger() right after it, so that at most one kernel waits behind the running one and its
+// blocks never compete with blocks of the running kernel that have not started yet.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 __device__ __forceinline__ float bf16_bits_to_float(uint32_t h) { return __uint_as_float(h << 16); }
 
 // 2^k for k in [-126, 127]

@@ -21,6 +21,8 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
     __shared__ float so[4][D];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int row = blockIdx.x * 4 + warp;           // b * Hq + hq
+    pdl_wait();
+    pdl_trigger();
     if (row >= n_rows) return;
     const int b = row / n_q_heads, hq = row % n_q_heads;
     int len = seq_lens[b];
@@ -211,9 +213,9 @@ kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype 
     else st = launch_decode_mma(a, s);
     if (st != KVBFP_OK) return st;
     const int n_rows = f.batch * n_q_heads;
-    lse_merge<<<(n_rows + 3) / 4, 128, 0, s>>>(a.partials, seq_lens, inv_perm_v, out, n_rows, n_q_heads, group,
-                                              a.n_chunks, a.chunk, a.len_cap, split.n_warps, split.item_tokens,
-                                              split.items_per_pair, split.range_items, split.range_extra);
+    (void)launch_pdl(lse_merge, dim3((n_rows + 3) / 4), dim3(128), 0, s, (const float*)a.partials, seq_lens, inv_perm_v, out,
+                     n_rows, n_q_heads, group, a.n_chunks, a.chunk, a.len_cap, split.n_warps, split.item_tokens,
+                     split.items_per_pair, split.range_items, split.range_extra);
     KVBFP_LAUNCH_CHECK("lse_merge");
     return KVBFP_OK;
 }

@@ -81,6 +81,8 @@ constexpr uint32_t kBias = 0xE488E488u;         // fp16 -1160.0 twice
 // the coefficients c1 = q_hi/16 (whole byte) and c2 = q_lo - q_hi/16 (low nibble), normalised per query
 // head by a power of two 2^qe, and qe itself.
 __global__ void __launch_bounds__(32) make_qfrag4(DecodeArgs a, int NT, int32_t* qmeta) {
+    pdl_wait();
+    pdl_trigger();
     const int N = a.fmt.block;
     const int lane = threadIdx.x, gp = lane >> 2, tp = lane & 3;
     const int item = blockIdx.x;
@@ -275,6 +277,8 @@ __device__ __forceinline__ QWord query_word(const DecodeArgs& a, float (&v)[8]) 
 // take the query heads (0, 1) of the n-tile, then (2, 3); all loads go out first.
 template <int N>
 __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_t* qmeta) {
+    pdl_wait();
+    pdl_trigger();
     constexpr int NBLK = D / N;
     const int lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int item = blockIdx.x * 4 + (threadIdx.x >> 5);
@@ -400,6 +404,8 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
     constexpr int NBLK = KI ? D / N : 1;              // blocks of a row (integer path)
     static_assert(!MHA || (KI && NT == 1), "the single-head path is built on the integer scores");
     extern __shared__ __align__(1024) uint8_t smem[];         // the swizzle pattern is a function of the address
+    pdl_wait();
+    pdl_trigger();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
@@ -1050,10 +1056,10 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
                                                (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
     if (N < 32) {
-        make_qfrag4<<<n_pre, 32, 0, s>>>(a, NT, qmeta);
+        (void)launch_pdl(make_qfrag4, dim3(n_pre), dim3(32), 0, s, a, NT, qmeta);
         KVBFP_LAUNCH_CHECK("make_qfrag4");
     } else if (!MHA) {    // (with one query head per kv head the main kernel forms the query coefficients itself)
-        make_qfrag4i<(N >= 32 ? N : 32)><<<(n_pre + 3) / 4, 128, 0, s>>>(a, NT, qmeta);
+        (void)launch_pdl(make_qfrag4i<(N >= 32 ? N : 32)>, dim3((n_pre + 3) / 4), dim3(128), 0, s, a, NT, qmeta);
         KVBFP_LAUNCH_CHECK("make_qfrag4i");
     }
     DecodeArgs b;
@@ -1077,7 +1083,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma4<N, NT, MHA><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b, qmeta, k_map, v_map);
+    (void)launch_pdl(decode_mma4<N, NT, MHA>, dim3(grid), dim3(kWarps * 32), G_::SMEM_BYTES, s, b, (const int32_t*)qmeta, k_map, v_map);
     KVBFP_LAUNCH_CHECK("decode_mma4");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;

@@ -77,6 +77,8 @@ struct Geo6 {
 
 template <int N>
 __global__ void __launch_bounds__(kWarps * 32, kMinCtas) decode_mma6(DecodeArgs a) {
+    pdl_wait();
+    pdl_trigger();
     using G_ = Geo6<N>;
     constexpr int ROW_E = G_::ROW_E;
     constexpr int NBLK = D / N;                       // blocks of a row
@@ -553,7 +555,7 @@ kvbfp_status launch2(const DecodeArgs& a, cudaStream_t s, Split* split) {
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma6<N><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b);
+    (void)launch_pdl(decode_mma6<N>, dim3(grid), dim3(kWarps * 32), G_::SMEM_BYTES, s, b);
     KVBFP_LAUNCH_CHECK("decode_mma6");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;

@@ -48,6 +48,8 @@ constexpr uint32_t kBias = 0xE480E480u;         // fp16 -1152.0 twice
 // g = (query g/2, digit g%2: 0 = d1, 1 = d0).  qmeta[query][2 blk] = scale * log2(e) * 2^(qe - 14) as float bits,
 // qmeta[query][2 blk + 1] = 128 * sum(C) of the block.
 __global__ void __launch_bounds__(128) make_qfrag8i(DecodeArgs a, int NT, int32_t* qmeta) {
+    pdl_wait();
+    pdl_trigger();
     const int N = a.fmt.block, nblk = D / N;
     const int s = threadIdx.x, blk = s / N;
     const int item = blockIdx.x;
@@ -146,6 +148,8 @@ struct Geo8 {
 
 template <int N, int NT>
 __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, const int32_t* __restrict__ qmeta) {
+    pdl_wait();
+    pdl_trigger();
     using G_ = Geo8<N>;
     constexpr int ROW_E = G_::ROW_E;
     constexpr int NBLK = D / N;                       // blocks of a row
@@ -531,7 +535,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     int32_t* qmeta = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(a.qfrag) +
                                                (size_t)a.fmt.batch * a.fmt.n_kv_heads * NT * 8 * 32 * 2 * sizeof(uint32_t));
     const int n_pre = a.fmt.batch * a.fmt.n_kv_heads * NT;
-    make_qfrag8i<<<n_pre, 128, 0, s>>>(a, NT, qmeta);
+    (void)launch_pdl(make_qfrag8i, dim3(n_pre), dim3(128), 0, s, a, NT, qmeta);
     KVBFP_LAUNCH_CHECK("make_qfrag8i");
     DecodeArgs b;
     int grid = 0;
@@ -540,7 +544,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    decode_mma8<N, NT><<<grid, kWarps * 32, G_::SMEM_BYTES, s>>>(b, qmeta);
+    (void)launch_pdl(decode_mma8<N, NT>, dim3(grid), dim3(kWarps * 32), G_::SMEM_BYTES, s, b, (const int32_t*)qmeta);
     KVBFP_LAUNCH_CHECK("decode_mma8");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;
