@@ -739,6 +739,41 @@ def test_rope_tables_and_apply(oracle, half_split):
         assert np.allclose(yb[r, 1], ref, rtol=2 ** -8, atol=1e-3)
 
 
+def test_rope_apply_runs_tiles_and_unpaired_tables(oracle):
+    """kvbfp_rope_apply over several row tiles: a run of positions that counts up (the tabulated turn from the
+    tile's first angle), with a ragged last tile, in f32 and bf16; and tables that do NOT pair the slots up
+    (partner map that is no involution, unrelated frequencies), which take the slot-by-slot form of Eq. (4)."""
+    rng = np.random.default_rng(31)
+    H, d, rows = 2, 128, 100
+    perm = np.stack([rng.permutation(d) for _ in range(H)]).astype(np.int32)
+    inv = np.argsort(perm, axis=1).astype(np.int32)
+    th, pa, sg = B.rope_tables(dev(torch.from_numpy(perm)), dev(torch.from_numpy(inv)), H, d, 10000.0, False)
+    t0, p0, s0 = oracle.rope_tables(d, 10000.0, False)
+    tabs = [oracle.rope_permute_tables(perm[h], inv[h], t0, p0, s0) for h in range(H)]
+    x = rng.standard_normal((rows, H, d)).astype(np.float32)
+    pos = (50000 + np.arange(rows)).astype(np.int32)
+    y = host(B.rope_apply(dev(torch.from_numpy(x)), dev(torch.from_numpy(pos)), th, pa, sg)).astype(np.float64)
+    xb = torch.from_numpy(x).to(torch.bfloat16)
+    yb = host(B.rope_apply(dev(xb), dev(torch.from_numpy(pos)), th, pa, sg).float()).astype(np.float64)
+    for h in range(H):
+        for r in range(rows):
+            ref = oracle.rope_apply(x[r, h].astype(np.float64), float(pos[r]), *tabs[h])
+            assert np.allclose(y[r, h], ref, rtol=0, atol=2e-6)
+            refb = oracle.rope_apply(xb[r, h].float().numpy().astype(np.float64), float(pos[r]), *tabs[h])
+            assert np.allclose(yb[r, h], refb, rtol=2 ** -8, atol=1e-3)
+    # free tables
+    th_f = rng.uniform(1e-4, 1.0, size=(H, d))
+    pa_f = rng.integers(0, d, size=(H, d)).astype(np.int32)
+    sg_f = rng.choice([-1.0, 1.0], size=(H, d)).astype(np.float32)
+    pos_f = np.concatenate([np.arange(70), rng.integers(0, 90000, size=30)]).astype(np.int32)
+    yf = host(B.rope_apply(dev(torch.from_numpy(x)), dev(torch.from_numpy(pos_f)), dev(torch.from_numpy(th_f)),
+                           dev(torch.from_numpy(pa_f)), dev(torch.from_numpy(sg_f)))).astype(np.float64)
+    for h in range(H):
+        for r in range(rows):
+            ref = oracle.rope_apply(x[r, h].astype(np.float64), float(pos_f[r]), th_f[h], pa_f[h], sg_f[h].astype(np.float64))
+            assert np.allclose(yf[r, h], ref, rtol=0, atol=3e-6)
+
+
 # ------------------------------------------------------------------------------- full-size workloads
 @pytest.mark.parametrize("half_split", [False, True])
 @pytest.mark.parametrize("p,n", [(4, 32), (4, 16), (8, 128), (6, 64)])
