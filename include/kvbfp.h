@@ -316,7 +316,8 @@ kvbfp_status kvbfp_selftest_wait_timeout(uint32_t tries, uint32_t hint_ns, void*
  * the merge finds those partial results again with the same integer arithmetic.  These calls expose that arithmetic
  * as the kernels use it, so that it can be checked on its own.
  *   kvbfp_split_plan         for `pairs` pairs of at most `len_cap` tokens in chunks of `chunk` tokens (a multiple of
- *                            128), items of `fine_tokens` tokens where the plan allows them, on a device that holds
+ *                            128), items of `fine_tokens` tokens (a multiple of 16 that divides the chunk; the
+ *                            kernels ask for 64) where the plan allows them, on a device that holds
  *                            `capacity_blocks` thread blocks of `warps_per_block` warps:
  *                            out6 = {grid, n_warps, item_tokens, items_per_pair, range_items, range_extra}
  *   kvbfp_split_range_start  first item of range w (the first range_extra ranges hold range_items + 1 items)

@@ -59,30 +59,42 @@ __host__ __device__ __forceinline__ int range_of(int x, int range_items, int ran
     return x < big ? x / (range_items + 1) : range_extra + (x - big) / range_items;
 }
 // Slot (chunk-sized, n_chunks per pair) that receives the partial of a run whose first item within its pair
-// is `item`.  Items are whole chunks, or half chunks: then two runs can start in the first chunk of a pair (one
-// that holds only item 0, the next from item 1 on), so odd items round up; ranges hold four items or more, so
-// no other two runs start within two items of each other and the clamp at the last slot is safe as well --
-// provided a pair has two slots or more: with a single chunk per pair, items 0 and 1 would share slot 0, so
-// plan_persistent() never cuts such pairs into half chunks.
+// is `item`.  Items are whole chunks, or chunk / R tokens with R = 2 or more: then slot = ceil(item / R), at most
+// the last one.  Runs of a pair start at item 0 and at range boundaries, which lie a whole range apart: with ranges
+// of 2R - 1 items or more, two starts never round up to the same slot, and a start that is clamped to the last slot
+// (item > (n_chunks - 1) R) has its predecessor at or below (n_chunks - 2) R, i.e. in an earlier slot -- provided a
+// pair has two slots or more: with a single chunk per pair every start would share slot 0, so plan_persistent()
+// never cuts such pairs finer than chunks.
 __host__ __device__ __forceinline__ int partial_slot(int item, int item_tokens, int chunk, int n_chunks) {
     if (item_tokens == chunk) return item;
-    const int s = (item + 1) >> 1;
+    const int R = chunk / item_tokens;
+    const int s = (item + R - 1) / R;
     return s < n_chunks ? s : n_chunks - 1;
 }
-// Work split of a persistent kernel (host side).  Items are pieces of `fine_tokens` tokens (half a chunk) when the
-// library chose the chunking (chunk == kMinChunk == 2 * fine_tokens), a pair has two chunks or more, and every warp
-// still gets five or more items on average, so four at the least (the ranges then differ by one piece of work at
-// most and partial_slot() keeps the runs' partial results apart); whole chunks otherwise.  The items are cut into one contiguous range per warp
-// of min(capacity, blocks needed) thread blocks.  Fills the range fields of `b` and `split`, returns the grid.
+// Work split of a persistent kernel (host side).  Items are pieces of fine_tokens tokens (chunk / R, a multiple of the
+// 16 tokens that copies start on) when the library chose the chunking (chunk == kMinChunk), a pair has two chunks or
+// more, and every warp still gets 2R + 1 or more items on average, so 2R at the least (partial_slot() then keeps the
+// runs' partial results apart); whole chunks otherwise.  The kernels ask for kItemTokens = 64, their tile: with
+// 16-token items the ranges come out more evenly (two warps then differ by a quarter of a tile, not a whole one), but
+// every run then ends in a partial tile that is copied and worked on like a whole one, and the launch was 1-2 %
+// slower.  The items are cut into one contiguous range per warp of min(capacity, blocks needed) thread blocks.
+// Fills the range fields of `b` and `split`, returns the grid.
+constexpr int kItemTokens = 64;
 inline kvbfp_status plan_persistent(const DecodeArgs& a, int fine_tokens, int capacity_blocks, int warps_per_block,
                                     DecodeArgs* b, Split* split, int* grid) {
     *b = a;
     const int64_t pairs = (int64_t)a.fmt.batch * a.fmt.n_kv_heads;
-    const int fine_per_pair = (a.len_cap + fine_tokens - 1) / fine_tokens;
-    const bool fine = a.chunk == 2 * fine_tokens && a.chunk == kMinChunk && a.n_chunks >= 2 &&
-                      pairs * fine_per_pair >= 5LL * capacity_blocks * warps_per_block;
-    b->item_tokens = fine ? fine_tokens : a.chunk;
-    b->items_per_pair = fine ? fine_per_pair : a.n_chunks;
+    b->item_tokens = a.chunk;
+    b->items_per_pair = a.n_chunks;
+    if (fine_tokens >= 16 && fine_tokens % 16 == 0 && fine_tokens < a.chunk && a.chunk % fine_tokens == 0) {   // (copies start on 16-token groups)
+        const int R = a.chunk / fine_tokens;
+        const int fine_per_pair = (a.len_cap + fine_tokens - 1) / fine_tokens;
+        if (a.chunk == kMinChunk && a.n_chunks >= 2 &&
+            pairs * fine_per_pair >= (int64_t)(2 * R + 1) * capacity_blocks * warps_per_block) {
+            b->item_tokens = fine_tokens;
+            b->items_per_pair = fine_per_pair;
+        }
+    }
     const int64_t n_items = pairs * b->items_per_pair;
     if (n_items >= (int64_t)1 << 31) return KVBFP_ERR_UNSUPPORTED;         // item indices are 32-bit in the kernels
     const int64_t want = (n_items + warps_per_block - 1) / warps_per_block;

@@ -1064,7 +1064,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     }
     DecodeArgs b;
     int grid = 0;
-    const kvbfp_status st = plan_persistent(a, kTile, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
+    const kvbfp_status st = plan_persistent(a, kItemTokens, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
     if (st != KVBFP_OK) return st;
     // tensor maps of the two mantissa planes (this device's memory; rows of two tokens, boxes of kTile tokens)
     // (a decode loop passes the same planes step after step: the last pair of maps is kept per host thread)

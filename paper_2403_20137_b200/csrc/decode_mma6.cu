@@ -550,7 +550,7 @@ kvbfp_status launch2(const DecodeArgs& a, cudaStream_t s, Split* split) {
     }
     DecodeArgs b;
     int grid = 0;
-    const kvbfp_status st = plan_persistent(a, kTile, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
+    const kvbfp_status st = plan_persistent(a, kItemTokens, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
     if (st != KVBFP_OK) return st;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);

@@ -32,7 +32,6 @@ constexpr int kWarps = 4;
 constexpr int kMT = 2;                  // 16-token MMA row tiles per stage
 constexpr int kTile = 16 * kMT;         // tokens per stage
 constexpr int kStages = 2;
-constexpr int kItemFine = 64;           // tokens per work item when the library chose the chunking (half a chunk)
 constexpr int D = kHeadDim;
 constexpr int ROW_M = D;                // one byte per slot
 constexpr int kTopShift = 5;            // weight of a block at the reference exponent is 2^kTopShift
@@ -539,7 +538,7 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     KVBFP_LAUNCH_CHECK("make_qfrag8i");
     DecodeArgs b;
     int grid = 0;
-    const kvbfp_status st = plan_persistent(a, kItemFine, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
+    const kvbfp_status st = plan_persistent(a, kItemTokens, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
     if (st != KVBFP_OK) return st;
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);

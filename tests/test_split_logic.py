@@ -62,8 +62,9 @@ def check_case(pairs, len_cap, fine_tokens, capacity_blocks, warps_per_block, ch
     it, ipp = p["item_tokens"], p["items_per_pair"]
     assert it in (fine_tokens, chunk) and ipp == (len_cap + it - 1) // it
     assert p["n_warps"] == p["grid"] * warps_per_block and 1 <= p["grid"] <= capacity_blocks
-    if it != chunk:                       # half-chunk items: only where the slots of a pair can stay distinct
-        assert n_chunks >= 2 and p["range_items"] >= 4
+    if it != chunk:                       # items of chunk / R tokens: only where the slots of a pair can stay distinct
+        R = chunk // it
+        assert chunk % it == 0 and it % 16 == 0 and n_chunks >= 2 and p["range_items"] >= 2 * R
     by_pair = {}
     for pr, c0, cnt in kernel_runs(p, pairs):
         by_pair.setdefault(pr, []).append(c0)
@@ -78,40 +79,43 @@ def check_case(pairs, len_cap, fine_tokens, capacity_blocks, warps_per_block, ch
 
 
 def test_small_shapes_exhaustively():
-    """One to four chunks per pair with both parities of the half-chunk count, every pair count that matters
-    around the point where the plan switches to half-chunk items, and several device sizes."""
+    """One to four chunks per pair with ragged and full last chunks, every pair count that matters around the
+    points where the plan switches to items of half a chunk and of an eighth of a chunk, and several device sizes."""
     fine_seen = coarse_seen = 0
     pair_counts = [1, 2, 3, 4, 5, 7, 10, 13, 16, 23, 31, 47, 64, 97, 128, 211, 300]
     for n_chunks in (1, 2, 3, 4):
         for len_cap in (128 * n_chunks - 127, 128 * n_chunks - 64, 128 * n_chunks - 63, 128 * n_chunks):
             for blocks in (1, 2, 3, 5, 8, 13):
                 for pairs in pair_counts:
-                    p = check_case(pairs, len_cap, 64, blocks, 4)
-                    fine_seen += p["item_tokens"] == 64
-                    coarse_seen += p["item_tokens"] == 128
-    assert fine_seen > 100 and coarse_seen > 100
+                    for fine in (16, 32, 64):
+                        p = check_case(pairs, len_cap, fine, blocks, 4)
+                        fine_seen += p["item_tokens"] == fine
+                        coarse_seen += p["item_tokens"] == 128
+    assert fine_seen > 300 and coarse_seen > 300
 
 
 def test_single_chunk_pairs_are_never_cut_in_half():
-    """64 < len_cap <= 128 gives one slot per pair; two half-chunk items of one pair would both map to it, so
-    whatever the number of pairs the plan keeps whole chunks there."""
+    """64 < len_cap <= 128 gives one slot per pair; two finer items of one pair would both map to it, so whatever
+    the number of pairs the plan keeps whole chunks there."""
     for pairs in (5, 600, 4440, 5120, 20000):
         for len_cap in (65, 100, 128):
-            p = plan(pairs, len_cap, 64, 444, 4)
+            for fine in (16, 64):
+                assert plan(pairs, len_cap, fine, 444, 4)["item_tokens"] == 128
+            p = plan(pairs, len_cap, 16, 444, 4)
             assert p["item_tokens"] == 128 and p["items_per_pair"] == 1
-    check_case(5120, 128, 64, 444, 4)
+    check_case(5120, 128, 16, 444, 4)
 
 
 def test_large_shapes_randomly():
     rng = random.Random(7)
-    cases = [(512, 8192, 64, 444, 4), (64, 32768, 64, 444, 4), (64, 32768, 64, 296, 4), (512, 8192, 32, 444, 4),
-             (3, 7 * 128, 64, 2, 4), (1, 1, 64, 444, 4)]
+    cases = [(512, 8192, 16, 296, 4), (64, 32768, 16, 444, 4), (64, 32768, 64, 296, 4), (512, 8192, 32, 444, 4),
+             (512, 8192, 64, 444, 4), (3, 7 * 128, 16, 2, 4), (1, 1, 16, 444, 4)]
     for _ in range(60):
-        cases.append((rng.randint(1, 400), rng.randint(1, 70 * 128), rng.choice((32, 64)), rng.randint(1, 30),
+        cases.append((rng.randint(1, 400), rng.randint(1, 70 * 128), rng.choice((16, 32, 64)), rng.randint(1, 30),
                       rng.choice((1, 2, 4))))
     for c in cases:
         check_case(*c)
     # caller-chosen chunk sizes are never cut finer
     for chunk in (256, 1024):
-        p = check_case(40, 5000, 64, 7, 4, chunk=chunk)
+        p = check_case(40, 5000, 16, 7, 4, chunk=chunk)
         assert p["item_tokens"] == chunk
