@@ -38,9 +38,9 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": 139.7107, "block": 32, "mant_bits": 4, "sources_sha256": "4150584d59fb4e6dfe9bbea904393f29197eb74086a20132c689f81db83c0145"},
-           "decode_mma8": {"bytes_per_unit": 264.3797, "block": 32, "mant_bits": 8, "sources_sha256": "b046192e7c5e3a98d6a85d578ec3d6b246a370801a397c32a983adf595983b38"},
-           "decode_mma6": {"bytes_per_unit": 204.1416, "block": 32, "mant_bits": 6, "sources_sha256": "39e1112b89fe0d9c252ce3c6a67d3befa7219dd10d60dbf5d765bbe5919d4138"}}
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 141.1555, "block": 32, "mant_bits": 4, "sources_sha256": "bd6ec2b1734142e85f9264432e3830cb98e919f42729967dc3f169c6805c667e"},
+           "decode_mma8": {"bytes_per_unit": 265.8467, "block": 32, "mant_bits": 8, "sources_sha256": "ce92d384364e96d75f25fab0ca6389f36a5c9eb96cf74c20af3345e1c2e2ea48"},
+           "decode_mma6": {"bytes_per_unit": 201.9604, "block": 32, "mant_bits": 6, "sources_sha256": "e385689f1c1aff6b9bdb23abdf17dfb4a6084e5568df0316cddb698466b03893"}}
 KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],
                   "decode_mma8": ["paper_2403_20137_b200/csrc/decode_mma8.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],
                   "decode_mma6": ["paper_2403_20137_b200/csrc/decode_mma6.cu", "paper_2403_20137_b200/csrc/ptx.cuh"]}
