@@ -498,9 +498,8 @@ def main():
     hout = torch.empty(Bn, Hq, d, dtype=torch.float32).pin_memory()
     staging = torch.empty(B.step_staging_bytes(rig.cache.fmt, Hq, rig.q.dtype), dtype=torch.uint8, device=dev)
 
-    def step_host():
-        B.decode_step_host(rig.cache, hk, hv, hq, rig.start_pos, rig.seq_lens, hout, staging, rig.ws, perm_k=rig.perm_k,
-                           max_len_hint=S, impl=rig.impl)
+    step_host = B.HostStep(rig.cache, hk, hv, hq, rig.start_pos, rig.seq_lens, hout, staging, rig.ws, perm_k=rig.perm_k,
+                           max_len_hint=S, impl=rig.impl)       # the arguments of the loop's call, marshalled once
 
     n_e2e = 0 if args.no_e2e else args.steps
     for _ in range(args.warmup if n_e2e else 0):

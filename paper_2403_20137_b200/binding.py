@@ -296,22 +296,44 @@ def step_staging_bytes(fmt, n_q_heads, dtype):
     return int(lib().kvbfp_step_staging_bytes(C.byref(fmt), n_q_heads, BF16 if dtype == torch.bfloat16 else F32))
 
 
+class HostStep:
+    """kvbfp_decode_step_host with its arguments marshalled once, for a decode loop that keeps its buffers: host
+    tensors k_new, v_new [B,1,H_kv,d], q [B,H_q,d] and the f32 output are refilled / read in place between calls,
+    start_pos and seq_lens are device tensors updated in place.  Calling the object runs one step and returns the
+    output tensor after the stream has been synchronised."""
+
+    def __init__(self, cache, k_new_host, v_new_host, q_host, start_pos, seq_lens, out_host, staging, workspace,
+                 perm_k=None, perm_v=None, inv_perm_v=None, softmax_scale=0.0, max_len_hint=0, impl=DECODE_AUTO,
+                 stream=None):
+        for t in (k_new_host, v_new_host, q_host, out_host):
+            if t.is_cuda or not t.is_contiguous():
+                raise ValueError("expected contiguous host tensors")
+        self.out_host = out_host
+        self._cs = cache.struct()
+        self._keep = (cache, k_new_host, v_new_host, q_host, start_pos, seq_lens, out_host, staging, workspace, perm_k,
+                      perm_v, inv_perm_v, stream)
+        self._fn = lib().kvbfp_decode_step_host
+        self._args = (C.byref(self._cs), _ptr(k_new_host), _ptr(v_new_host), _ptr(q_host), _dt(q_host), q_host.shape[1],
+                      _ptr(_dev(start_pos, torch.int32)), _ptr(_dev(seq_lens, torch.int32)), max_len_hint,
+                      _ptr(_dev(perm_k, torch.int32)), _ptr(_dev(perm_v, torch.int32)),
+                      _ptr(_dev(inv_perm_v, torch.int32)), float(softmax_scale), _ptr(out_host), _ptr(staging),
+                      staging.numel(), _ptr(workspace), workspace.numel(), impl, _stream(stream))
+
+    def __call__(self):
+        rc = self._fn(*self._args)
+        if rc != OK:
+            _check(rc)
+        return self.out_host
+
+
 def decode_step_host(cache, k_new_host, v_new_host, q_host, start_pos, seq_lens, out_host, staging, workspace,
                      perm_k=None, perm_v=None, inv_perm_v=None, softmax_scale=0.0, max_len_hint=0,
                      impl=DECODE_AUTO, stream=None):
     """kvbfp_decode_step_host: host tensors in (k_new, v_new [B,1,H_kv,d]; q [B,H_q,d]), host f32 out;
-    returns after the stream has been synchronised."""
-    for t in (k_new_host, v_new_host, q_host, out_host):
-        if t.is_cuda or not t.is_contiguous():
-            raise ValueError("expected contiguous host tensors")
-    cs = cache.struct()
-    _check(lib().kvbfp_decode_step_host(
-        C.byref(cs), _ptr(k_new_host), _ptr(v_new_host), _ptr(q_host), _dt(q_host), q_host.shape[1],
-        _ptr(_dev(start_pos, torch.int32)), _ptr(_dev(seq_lens, torch.int32)), max_len_hint,
-        _ptr(_dev(perm_k, torch.int32)), _ptr(_dev(perm_v, torch.int32)), _ptr(_dev(inv_perm_v, torch.int32)),
-        float(softmax_scale), _ptr(out_host), _ptr(staging), staging.numel(), _ptr(workspace), workspace.numel(),
-        impl, _stream(stream)))
-    return out_host
+    returns after the stream has been synchronised.  (One call; a loop over fixed buffers keeps a HostStep.)"""
+    return HostStep(cache, k_new_host, v_new_host, q_host, start_pos, seq_lens, out_host, staging, workspace,
+                    perm_k=perm_k, perm_v=perm_v, inv_perm_v=inv_perm_v, softmax_scale=softmax_scale,
+                    max_len_hint=max_len_hint, impl=impl, stream=stream)()
 
 
 def profile_decode_events(start=None, stop=None):

@@ -564,7 +564,7 @@ def test_decode_step_host_equals_device_path(oracle, cfg, pinned):
     B.append(caches[0], dev(kn), dev(vn), sp, perm_k=perm)
     ref = B.decode_attn(caches[0], dev(q), lens, perm_k=perm)
     pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
-    hk, hv, hq = pin(kn), pin(vn), pin(q.contiguous())
+    hk, hv, hq = pin(kn), pin(vn), pin(q.clone())
     hout = pin(torch.zeros(Bn, w.n_q_heads, 128, dtype=torch.float32))
     staging = torch.empty(B.step_staging_bytes(caches[1].fmt, w.n_q_heads, q.dtype), dtype=torch.uint8, device="cuda")
     ws = torch.empty(B.decode_workspace_bytes(caches[1].fmt, w.n_q_heads), dtype=torch.uint8, device="cuda")
@@ -573,6 +573,13 @@ def test_decode_step_host_equals_device_path(oracle, cfg, pinned):
         assert torch.equal(hout, ref.cpu())
     for name in ("k_mant", "k_exp", "v_mant", "v_exp"):
         assert torch.equal(getattr(caches[0], name), getattr(caches[1], name)), name
+    # the same call with its arguments marshalled once, as a decode loop keeps it: the buffers are refilled in place
+    step = B.HostStep(caches[1], hk, hv, hq, sp, lens, hout, staging, ws, perm_k=perm)
+    hq.copy_(-q)
+    hout.zero_()
+    assert step() is hout
+    ref2 = B.decode_attn(caches[0], dev(-q), lens, perm_k=perm)
+    assert torch.equal(hout, ref2.cpu()) and not torch.equal(ref2, ref)
     assert B.device_status() == 0
 
 
