@@ -33,8 +33,8 @@ from paper_2403_20137_b200 import workloads as W  # noqa: E402
 METRIC = "decode_attn_tokens_per_s"
 UNIT = "tokens/s"
 
-# DRAM traffic of the dominant kernel from one ncu capture (profiles/decode_mma4_b4_s8192_ncu_full.md; the 8-bit
-# kernel: profiles/other_decode_kernels_b4_s8192_ncu_sections.md; the 6-bit one: profiles/decode_mma6_b4_s8192_ncu_sections.md):
+# DRAM traffic of the dominant kernel from one ncu capture per kernel (batch 4 of the same shape; the summaries of
+# those captures are kept under profiles/):
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
