@@ -1,7 +1,8 @@
 // Eq. (1) of the paper: stored mantissas times 2^e back to numbers, optionally in the original channel order.
 //
 // A thread block takes a tile of 64 token rows of one (batch, head): the packed rows are contiguous in their
-// plane and come in with 16-byte loads into shared memory; every thread then owns four output channels of a row
+// plane and come in with 16-byte loads into shared memory, the exponent bytes as the fp32 weights 2^(e - 127 - (p-2))
+// they stand for (worked out once per block of a row, not once per element); every thread then owns four output channels of a row
 // (so a warp writes one row with one 16-byte store per lane, fully coalesced) and picks the fields of those
 // channels out of the staged row -- with a permutation that is a gather through the inverse permutation, which
 // the block builds once in shared memory.  One launch covers any rectangle (sequences x heads x tokens).
@@ -41,7 +42,7 @@ template <int P, typename T, bool PERM>
 __global__ void __launch_bounds__(kThreads) dequant_tile(DequantArgs a) {
     constexpr int D = kHeadDim, ROW_M = D * P / 8;
     __shared__ __align__(16) uint8_t smant[kTileTok * ROW_M + 16];      // (+16: the two-byte read of the last field)
-    __shared__ uint8_t sexp[kTileTok * 8];
+    __shared__ float sw[kTileTok * 8];                                   // weight of one mantissa unit per (row, block)
     __shared__ int sinv[D];
     const int tid = threadIdx.x, lane = tid & 31, sub = tid >> 5;
     const int tile = blockIdx.x % a.tiles;
@@ -56,7 +57,7 @@ __global__ void __launch_bounds__(kThreads) dequant_tile(DequantArgs a) {
     const uint4* src = reinterpret_cast<const uint4*>(a.mant + row0 * ROW_M);
     for (int i = tid; i < rows * (ROW_M / 16); i += kThreads) reinterpret_cast<uint4*>(smant)[i] = __ldg(src + i);
     const uint8_t* esrc = a.exp8 + row0 * row_e;
-    for (int i = tid; i < rows * row_e; i += kThreads) sexp[i] = __ldg(esrc + i);
+    for (int i = tid; i < rows * row_e; i += kThreads) sw[i] = unit_weight(__ldg(esrc + i), P);
     if (PERM && tid < D) sinv[a.perm[h * D + tid] & (D - 1)] = tid;
     __syncthreads();
 
@@ -79,7 +80,7 @@ __global__ void __launch_bounds__(kThreads) dequant_tile(DequantArgs a) {
             uint32_t w = mrow[byte[j]];
             if (P == 6) w |= (uint32_t)mrow[byte[j] + 1] << 8;        // a 6-bit field may straddle two bytes
             const int m = (int)((w >> sh[j]) & ((1u << P) - 1u)) - (1 << (P - 1));
-            v[j] = (float)m * unit_weight(sexp[r * row_e + eb[j]], P);
+            v[j] = (float)m * sw[r * row_e + eb[j]];
         }
         store4<T>(out + (int64_t)(tok0 + r) * a.out_tok_stride, v[0], v[1], v[2], v[3]);
     }
