@@ -63,8 +63,9 @@ inline size_t row_e_bytes(const kvbfp_format& f) { return (size_t)(f.head_dim / 
 // stream serialization: the next kernel's thread blocks may become resident and run their set-up while the kernel
 // before it is still running.  Every such kernel calls pdl_wait() before its first access to global memory (it
 // returns once the kernel before it has completed and its writes are visible; at once if the launch had no such
-// predecessor) and pdl_trigger() right after it, so that at most one kernel waits behind the running one and its
-// blocks never compete with blocks of the running kernel that have not started yet.
+// predecessor) and pdl_trigger() after it, so that at most one kernel waits behind the running one and its blocks
+// never compete with blocks of the running kernel that have not started yet: the short kernels right after the
+// wait, the persistent decode kernels at their end (waiting blocks on an SM slow its streaming warps down).
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 

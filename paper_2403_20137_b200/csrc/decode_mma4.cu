@@ -405,7 +405,6 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
     static_assert(!MHA || (KI && NT == 1), "the single-head path is built on the integer scores");
     extern __shared__ __align__(1024) uint8_t smem[];         // the swizzle pattern is a function of the address
     pdl_wait();
-    pdl_trigger();
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
@@ -1025,6 +1024,9 @@ decode_mma4(DecodeArgs a, const int32_t* __restrict__ qmeta, const __grid_consta
         }
     }
 
+    // the merge kernel is released only here: its thread blocks, dispatched while this kernel still streams, slowed
+    // the SMs they landed on, and with one range per warp the slowest SM sets the time of the launch
+    pdl_trigger();
     if (timed_out) {
         // give the copies still in flight a bounded chance to land before the shared memory is released
         if (lane == 0) raise_flag(a.status, KVBFP_FLAG_WAIT_TIMEOUT);

@@ -78,7 +78,6 @@ struct Geo6 {
 template <int N>
 __global__ void __launch_bounds__(kWarps * 32, kMinCtas) decode_mma6(DecodeArgs a) {
     pdl_wait();
-    pdl_trigger();
     using G_ = Geo6<N>;
     constexpr int ROW_E = G_::ROW_E;
     constexpr int NBLK = D / N;                       // blocks of a row
@@ -523,6 +522,9 @@ __global__ void __launch_bounds__(kWarps * 32, kMinCtas) decode_mma6(DecodeArgs 
         }
     }
 
+    // the merge kernel is released only here: its thread blocks, dispatched while this kernel still streams, slowed
+    // the SMs they landed on, and with one range per warp the slowest SM sets the time of the launch
+    pdl_trigger();
     if (timed_out) {
         // give the copies still in flight a bounded chance to land before the shared memory is released
         if (lane == 0) raise_flag(a.status, KVBFP_FLAG_WAIT_TIMEOUT);

@@ -5,7 +5,10 @@
 //
 // Same launch design as the 4-bit kernel: work items laid out pair-major and cut into one contiguous range per
 // resident warp (persistent), "runs" with one partial result each, a private ring of shared-memory stages per
-// warp filled by 1-D bulk asynchronous copies (each warp fetches its own tiles), no block-wide barrier in the loop.
+// warp (each warp fetches its own tiles), no block-wide barrier in the loop.  The K and V byte tiles come by tiled 2-D
+// asynchronous copies over tensor maps of the two planes (a row = one token = 128 bytes, 128-byte swizzle: the
+// 16-byte piece p of row r lands at piece p ^ (r % 8)), which makes the fragment loads below conflict-free; the
+// exponent bytes come by 1-D bulk copies.
 //
 // A stored byte is B = M + 128 (excess code), so nothing has to be unpacked.
 //   Scores: the bytes are the unsigned operand of a byte MMA.  The query block is cast to 15-bit fixed point
@@ -130,30 +133,38 @@ __global__ void __launch_bounds__(128) make_qfrag8i(DecodeArgs a, int NT, int32_
 }
 
 // ------------------------------------------------------------------ main kernel
+constexpr int kTileBytes = kTile * ROW_M;      // 4 KiB: a whole number of 1 KiB swizzle periods
 template <int N>
 struct Geo8 {
     static constexpr int ROW_E = D / N;
+    // mantissa tiles first (1 KiB-aligned: the swizzle pattern is a function of the address), then the exponent bytes
+    static constexpr int MANT_STAGE = 2 * kTileBytes;                   // K tile, V tile
     static constexpr int KM_OFF = 0;
-    static constexpr int VM_OFF = kTile * ROW_M;
-    static constexpr int KE_OFF = 2 * kTile * ROW_M;
-    static constexpr int VE_OFF = KE_OFF + kTile * ROW_E;
-    static constexpr int STAGE_BYTES = 2 * kTile * (ROW_M + ROW_E);
-    static constexpr int WARP_BYTES = kStages * STAGE_BYTES;
-    static constexpr int LUT_OFF = kWarps * WARP_BYTES;                 // uint2[kLutEntries]
+    static constexpr int VM_OFF = kTileBytes;
+    static constexpr int EXP_OFF = kWarps * kStages * MANT_STAGE;       // per (warp, stage): K bytes, V bytes
+    static constexpr int EXP_STAGE = 2 * kTile * ROW_E;
+    static constexpr int KE_OFF = 0;
+    static constexpr int VE_OFF = kTile * ROW_E;
+    static constexpr int LUT_OFF = EXP_OFF + kWarps * kStages * EXP_STAGE;   // uint2[kLutEntries]
     static constexpr int LUTF_OFF = LUT_OFF + kLutEntries * 8;          // float[256]
     static constexpr int BAR_OFF = LUTF_OFF + 256 * 4;
     static constexpr int SMEM_BYTES = BAR_OFF + kWarps * kStages * 8;
 };
+// Tokens of a 16-token row tile whose V bytes lane (g, t) loads for P.V, k = 0..3: 2t, 2t+1, 2t+8, 2t+9 -- the MMA's
+// own order of the contraction index, and rows whose numbers mod 8 differ in bits 1 and 2 across t, so that the
+// eight lanes of a quarter warp (two values of g, four of t) read eight different swizzled pieces.
+__device__ __forceinline__ int tok8(int t, int k) { return 2 * t + (k & 1) + 4 * (k & 2); }
 
 template <int N, int NT>
-__global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, const int32_t* __restrict__ qmeta) {
+__global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, const int32_t* __restrict__ qmeta,
+                                                              const __grid_constant__ CUtensorMap k_map,
+                                                              const __grid_constant__ CUtensorMap v_map) {
     pdl_wait();
-    pdl_trigger();
     using G_ = Geo8<N>;
     constexpr int ROW_E = G_::ROW_E;
     constexpr int NBLK = D / N;                       // blocks of a row
     constexpr int GRP_PER_BLK = 4 / NBLK;             // 32-byte groups per block
-    extern __shared__ __align__(128) uint8_t smem[];
+    extern __shared__ __align__(1024) uint8_t smem[];         // the swizzle pattern is a function of the address
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t = lane & 3;
     const int Hkv = a.fmt.n_kv_heads, Gq = a.n_q_heads / Hkv;
@@ -184,8 +195,13 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
         return r;
     };
 
-    uint8_t* wsm = smem + warp * G_::WARP_BYTES;
-    const uint32_t wsm_u32 = smem_u32(wsm);
+    if (smem_u32(smem) & 1023u) {        // never expected: the tiles would be read with the wrong pattern
+        if (threadIdx.x == 0) raise_flag(a.status, KVBFP_FLAG_WAIT_TIMEOUT);
+        return;                          // (the whole block, before any copy is issued)
+    }
+    uint8_t* wsm = smem + warp * kStages * G_::MANT_STAGE;                          // this warp's mantissa tiles
+    uint8_t* wse = smem + G_::EXP_OFF + warp * kStages * G_::EXP_STAGE;             // and exponent bytes
+    const uint32_t wsm_u32 = smem_u32(wsm), wse_u32 = smem_u32(wse);
     const uint32_t bar0 = smem_u32(smem + G_::BAR_OFF + warp * kStages * 8);
     if (lane == 0) {
 #pragma unroll
@@ -195,10 +211,13 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
     }
     __syncwarp();
 
-    // ---- producer: lanes 0..3 each own one of the four spans of a stage
-    const uint8_t* my_base = lane == 0 ? a.k_mant : lane == 1 ? a.v_mant : lane == 2 ? a.k_exp : a.v_exp;
-    const int my_row_bytes = (lane < 2) ? ROW_M : ROW_E;
-    const uint32_t my_dst = wsm_u32 + (lane == 0 ? G_::KM_OFF : lane == 1 ? G_::VM_OFF : lane == 2 ? G_::KE_OFF : G_::VE_OFF);
+    // ---- producer: lanes 0..3 each own one of the four pieces of a stage: the K and V byte tiles (tiled copies of
+    // kTile whole rows: rows past the sequence are never used, rows past the plane arrive as zeros) and the K and V
+    // exponent bytes (1-D copies of the 16-token groups that hold tokens)
+    const uint8_t* my_exp = lane == 2 ? a.k_exp : a.v_exp;
+    const CUtensorMap* my_map = lane == 0 ? &k_map : &v_map;
+    const uint32_t my_dst = lane < 2 ? wsm_u32 + (lane == 0 ? G_::KM_OFF : G_::VM_OFF)
+                                     : wse_u32 + (lane == 2 ? G_::KE_OFF : G_::VE_OFF);
     int p_next = i0;
     Run pr;
     pr.n_tiles = 0;
@@ -214,9 +233,10 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
             const int off = p_tile * kTile;
             const int rows = min(kTile, ((pr.n_tok + 15) & ~15) - off);    // whole 16-token groups; stays below max_seq
             const uint32_t bar = bar0 + 8 * stage;
-            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(2 * rows * (ROW_M + ROW_E)));
+            if (lane == 0) mbar_expect_tx(bar, (uint32_t)(2 * kTileBytes + 2 * rows * ROW_E));
             __syncwarp(0xfu);
-            bulk_g2s(my_dst + stage * G_::STAGE_BYTES, my_base + (pr.row0 + off) * my_row_bytes, rows * my_row_bytes, bar);
+            if (lane < 2) tensor_g2s_2d(my_dst + stage * G_::MANT_STAGE, my_map, 0, (int)(pr.row0 + off), bar);
+            else bulk_g2s(my_dst + stage * G_::EXP_STAGE, my_exp + (pr.row0 + off) * ROW_E, rows * ROW_E, bar);
         }
         ++p_tile;
     };
@@ -235,12 +255,20 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
     __syncthreads();
     if (i0 >= i1) return;
 
-    // per-lane byte offsets inside a stage
-    const int k_off = G_::KM_OFF + g * ROW_M + t * 8;
+    // per-lane byte offsets inside a stage (mantissa tiles swizzled: byte b of row r sits at b ^ ((r % 8) << 4))
+    int k_sw[4];                                               // this lane's eight bytes of each 32-byte group, rows g and g + 8
+#pragma unroll
+    for (int grp = 0; grp < 4; ++grp) k_sw[grp] = G_::KM_OFF + g * ROW_M + ((t * 8 + 32 * grp) ^ (g << 4));
     const int kei_off = G_::KE_OFF + g * ROW_E;
-    const int v_off = G_::VM_OFF + t * ROW_M + g * 16;
-    const int ve_off = G_::VE_OFF + t * ROW_E + (16 * g) / N;
-    const int src_lo = 4 * t + (g >> 1), src_hi = 4 * (t + 4) + (g >> 1);
+    int v_off[4], ve_off[4];                                   // bytes [16g, 16g + 16) of rows tok8(t, k)
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int r = tok8(t, k);
+        v_off[k] = G_::VM_OFF + r * ROW_M + ((g ^ (r & 7)) << 4);
+        ve_off[k] = G_::VE_OFF + r * ROW_E + (16 * g) / N;
+    }
+    // softmax weights travel from the lanes that computed them (token = lane / 4 and + 8, column pair = lane % 4)
+    const int src_lo = 4 * tok8(t, 0) + (g >> 1), src_hi = 4 * tok8(t, 1) + (g >> 1);
     const uint32_t half_sel = (g & 1) ? 0x7632u : 0x5410u;     // odd columns carry the lo halves
 
     int stage = 0;
@@ -290,11 +318,11 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
         for (int nt = 0; nt < NT; ++nt) { m_run[nt] = -INFINITY; l_run[nt] = 0.f; }
 
         constexpr int VE_WORDS = kTile * ROW_E / 4;      // V exponent bytes of a stage, in words
-        auto raise_dv = [&](const uint8_t* st, int n_live) {
+        auto raise_dv = [&](const uint8_t* se, int n_live) {
             const int n_bytes = min(n_live, kTile) * ROW_E;
             uint32_t m = 0;
             for (int w = lane; w < VE_WORDS; w += 32) {
-                uint32_t x = *reinterpret_cast<const uint32_t*>(st + G_::VE_OFF + 4 * w);
+                uint32_t x = *reinterpret_cast<const uint32_t*>(se + G_::VE_OFF + 4 * w);
                 const int left = n_bytes - 4 * w;
                 if (left < 4) x = left <= 0 ? 0u : (x & ((1u << (8 * left)) - 1u));
                 m = vmaxu4(m, x);
@@ -320,7 +348,7 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
         };
 
         // one stage of kTile tokens; FULL = every row of the tile exists
-        auto tile_body = [&](const uint8_t* st, int n_live, auto full_tag) {
+        auto tile_body = [&](const uint8_t* st, const uint8_t* se, int n_live, auto full_tag) {
             constexpr bool FULL = decltype(full_tag)::value;
             if (FULL) {
                 uint32_t f = 0;
@@ -328,13 +356,13 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
                 for (int i = 0; i < (VE_WORDS + 31) / 32; ++i) {
                     const int w = lane + 32 * i;
                     if (VE_WORDS % 32 == 0 || w < VE_WORDS) {
-                        const uint32_t x = *reinterpret_cast<const uint32_t*>(st + G_::VE_OFF + 4 * w);
+                        const uint32_t x = *reinterpret_cast<const uint32_t*>(se + G_::VE_OFF + 4 * w);
                         f |= ((x & 0x00FF00FFu) + dv_probe) | (prmt(x, 0u, 0x4341u) + dv_probe);
                     }
                 }
-                if (__any_sync(0xffffffffu, (f & 0x80008000u) != 0u)) raise_dv(st, n_live);
+                if (__any_sync(0xffffffffu, (f & 0x80008000u) != 0u)) raise_dv(se, n_live);
             } else {
-                raise_dv(st, n_live);         // rows past the end may hold anything: masked there
+                raise_dv(se, n_live);         // rows past the end may hold anything: masked there
             }
             // ---- scores ---------------------------------------------------------
             float sc[kMT][NT][2];
@@ -346,11 +374,11 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
                     continue;
                 }
                 int acc[NT][NBLK][4];
-                const uint8_t* pa = st + k_off + mt * 16 * ROW_M;
+                const uint8_t* pa = st + mt * 16 * ROW_M;
 #pragma unroll
                 for (int grp = 0; grp < 4; ++grp) {        // 32-byte groups of the row; this lane's eight bytes of each
-                    const uint2 wa = *reinterpret_cast<const uint2*>(pa + 32 * grp);
-                    const uint2 wb = *reinterpret_cast<const uint2*>(pa + 8 * ROW_M + 32 * grp);
+                    const uint2 wa = *reinterpret_cast<const uint2*>(pa + k_sw[grp]);
+                    const uint2 wb = *reinterpret_cast<const uint2*>(pa + 8 * ROW_M + k_sw[grp]);
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         if (grp % GRP_PER_BLK == 0)   // first MMA of a block: the offsets' constant contribution goes in as C
@@ -365,8 +393,8 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
                 for (int nt = 0; nt < NT; ++nt) s0[nt] = s1[nt] = 0.f;
 #pragma unroll
                 for (int k = 0; k < NBLK; ++k) {
-                    const float w0 = lutf[st[kei_off + mt * 16 * ROW_E + k]];
-                    const float w1 = lutf[st[kei_off + (mt * 16 + 8) * ROW_E + k]];
+                    const float w0 = lutf[se[kei_off + mt * 16 * ROW_E + k]];
+                    const float w1 = lutf[se[kei_off + (mt * 16 + 8) * ROW_E + k]];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         const float f0 = __int2float_rn(256 * acc[nt][k][0] + acc[nt][k][1]);
@@ -418,7 +446,7 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
 #pragma unroll
             for (int mt = 0; mt < kMT; ++mt) {
                 if (!FULL && mt * 16 >= n_live) continue;
-                // B fragment of P^T for lane (g, t): column g = (query g/2, half g%2); tokens t, t+4 | t+8, t+12
+                // B fragment of P^T for lane (g, t): column g = (query g/2, half g%2); tokens 2t, 2t+1 | 2t+8, 2t+9
                 uint32_t pb[NT][2];
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt) {
@@ -428,25 +456,25 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
                     const float h0 = __uint_as_float(__float_as_uint(p0) & 0xffffe000u);
                     const float h1 = __uint_as_float(__float_as_uint(p1) & 0xffffe000u);
                     const uint32_t w0 = pack_f16x2_rn(h0, p0 - h0), w1 = pack_f16x2_rn(h1, p1 - h1);
-                    const uint32_t v0 = __shfl_sync(0xffffffffu, w0, src_lo);   // token t
-                    const uint32_t v1 = __shfl_sync(0xffffffffu, w0, src_hi);   // token t+4
-                    const uint32_t v2 = __shfl_sync(0xffffffffu, w1, src_lo);   // token t+8
-                    const uint32_t v3 = __shfl_sync(0xffffffffu, w1, src_hi);   // token t+12
+                    const uint32_t v0 = __shfl_sync(0xffffffffu, w0, src_lo);   // token 2t
+                    const uint32_t v1 = __shfl_sync(0xffffffffu, w0, src_hi);   // token 2t+1
+                    const uint32_t v2 = __shfl_sync(0xffffffffu, w1, src_lo);   // token 2t+8
+                    const uint32_t v3 = __shfl_sync(0xffffffffu, w1, src_hi);   // token 2t+9
                     pb[nt][0] = prmt(v0, v1, half_sel);
                     pb[nt][1] = prmt(v2, v3, half_sel);
                 }
-                // V pieces: bytes [16g, 16g+16) (slots 16g..16g+15) of tokens t, t+4, t+8, t+12 of this row tile
+                // V pieces: bytes [16g, 16g+16) (slots 16g..16g+15) of tokens tok8(t, 0..3) of this row tile
                 uint4 vw[4];
                 uint2 lv[4];
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    vw[k] = *reinterpret_cast<const uint4*>(st + v_off + (mt * 16 + 4 * k) * ROW_M);
-                    lv[k] = lutv[st[ve_off + (mt * 16 + 4 * k) * ROW_E]];
+                    vw[k] = *reinterpret_cast<const uint4*>(st + v_off[k] + mt * 16 * ROW_M);
+                    lv[k] = lutv[se[ve_off[k] + mt * 16 * ROW_E]];
                 }
                 if (!FULL) {       // rows past the end contribute exactly zero
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        if (mt * 16 + t + 4 * k >= n_live) lv[k] = make_uint2(0u, 0u);
+                        if (mt * 16 + tok8(t, k) >= n_live) lv[k] = make_uint2(0u, 0u);
                 }
                 const uint32_t sA = prmt(lv[0].x, lv[1].x, 0x7610u), cA = prmt(lv[0].y, lv[1].y, 0x7610u);
                 const uint32_t sB = prmt(lv[2].x, lv[3].x, 0x7610u), cB = prmt(lv[2].y, lv[3].y, 0x7610u);
@@ -470,10 +498,11 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
 
         for (int it = 0; it < cr.n_tiles; ++it) {
             if (!mbar_wait_bounded(bar0 + 8 * stage, parity)) { timed_out = true; break; }
-            const uint8_t* st = wsm + stage * G_::STAGE_BYTES;
+            const uint8_t* st = wsm + stage * G_::MANT_STAGE;
+            const uint8_t* se = wse + stage * G_::EXP_STAGE;
             const int n_live = cr.n_tok - it * kTile;        // tokens of this tile that exist (may exceed kTile)
-            if (n_live >= kTile) tile_body(st, n_live, std::true_type{});
-            else tile_body(st, n_live, std::false_type{});
+            if (n_live >= kTile) tile_body(st, se, n_live, std::true_type{});
+            else tile_body(st, se, n_live, std::false_type{});
             __syncwarp();
             issue_next(stage);
             if (++stage == kStages) { stage = 0; parity ^= 1u; }
@@ -505,6 +534,9 @@ __global__ void __launch_bounds__(kWarps * 32, 3) decode_mma8(DecodeArgs a, cons
         }
     }
 
+    // the merge kernel is released only here: its thread blocks, dispatched while this kernel still streams, slowed
+    // the SMs they landed on, and with one range per warp the slowest SM sets the time of the launch
+    pdl_trigger();
     if (timed_out) {
         // give the copies still in flight a bounded chance to land before the shared memory is released
         if (lane == 0) raise_flag(a.status, KVBFP_FLAG_WAIT_TIMEOUT);
@@ -540,10 +572,22 @@ kvbfp_status launch3(const DecodeArgs& a, cudaStream_t s, Split* split) {
     int grid = 0;
     const kvbfp_status st = plan_persistent(a, kItemTokens, resident[dev].load(std::memory_order_relaxed), kWarps, &b, split, &grid);
     if (st != KVBFP_OK) return st;
+    // tensor maps of the two byte planes (this device's memory; rows of one token, boxes of kTile tokens); a decode
+    // loop passes the same planes step after step: the last pair of maps is kept per host thread
+    struct MapCache { const void *k = nullptr, *v = nullptr; uint64_t rows = 0; int dev = -1; CUtensorMap k_map, v_map; };
+    static thread_local MapCache mc;
+    const uint64_t n_rows = (uint64_t)a.fmt.batch * a.fmt.n_kv_heads * a.fmt.max_seq;
+    if (mc.k != a.k_mant || mc.v != a.v_mant || mc.rows != n_rows || mc.dev != dev) {
+        mc.k = nullptr;
+        kvbfp_status ms = make_row_map(&mc.k_map, a.k_mant, n_rows, ROW_M, kTile);
+        if (ms == KVBFP_OK) ms = make_row_map(&mc.v_map, a.v_mant, n_rows, ROW_M, kTile);
+        if (ms != KVBFP_OK) return ms;
+        mc.k = a.k_mant; mc.v = a.v_mant; mc.rows = n_rows; mc.dev = dev;
+    }
     cudaEvent_t ev0, ev1;
     profile_events(&ev0, &ev1);
     if (ev0) KVBFP_CUDA(cudaEventRecord(ev0, s));
-    (void)launch_pdl(decode_mma8<N, NT>, dim3(grid), dim3(kWarps * 32), G_::SMEM_BYTES, s, b, (const int32_t*)qmeta);
+    (void)launch_pdl(decode_mma8<N, NT>, dim3(grid), dim3(kWarps * 32), G_::SMEM_BYTES, s, b, (const int32_t*)qmeta, mc.k_map, mc.v_map);
     KVBFP_LAUNCH_CHECK("decode_mma8");
     if (ev1) KVBFP_CUDA(cudaEventRecord(ev1, s));
     return KVBFP_OK;
