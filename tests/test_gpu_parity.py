@@ -583,6 +583,49 @@ def test_decode_step_host_equals_device_path(oracle, cfg, pinned):
     assert B.device_status() == 0
 
 
+@pytest.mark.parametrize("cfg,p", [(3, 4), (4, 4), (4, 8), (3, 6)])
+def test_back_to_back_steps_equal_synchronised_steps(oracle, cfg, p):
+    """The kernels of a step are launched so that each may be set up while the one before it still runs; each waits
+    for its predecessor before it touches memory.  Twelve steps issued back to back (append of a new token, decode,
+    every step's output kept) must give bit for bit what the same calls give with the device synchronised after every
+    single call, cache planes included; the last output is also checked against the oracle."""
+    import dataclasses
+    w = dataclasses.replace(W.CONFIGS[cfg], mant_bits=p)
+    Bn, S0, steps = 3, 700, 12
+    k, v = W.make_kv(w, n_tokens=S0 + steps, batch=Bn)
+    q0 = W.make_q(w, batch=Bn)
+    qs = [torch.roll(q0, 5 * i, dims=-1) * (1.0 + 0.125 * i) for i in range(steps)]      # a different query every step
+    _, perm, _ = B.calibrate(dev(k.reshape(-1, w.n_kv_heads, 128)), w.n_kv_heads, 128)
+    z = dev(torch.zeros(Bn, dtype=torch.int32))
+    runs = []
+    for sync in (False, True):
+        c = B.Cache(Bn, w.n_kv_heads, 128, 720, w.block, p, fill=0)
+        ws = torch.empty(B.decode_workspace_bytes(c.fmt, w.n_q_heads), dtype=torch.uint8, device="cuda")
+        B.append(c, dev(k[:, :S0]), dev(v[:, :S0]), z, perm_k=perm)
+        kd, vd, qd = dev(k), dev(v), [dev(q) for q in qs]
+        sps = [dev(torch.full((Bn,), S0 + i, dtype=torch.int32)) for i in range(steps)]
+        lens = [dev(torch.full((Bn,), S0 + i + 1, dtype=torch.int32)) for i in range(steps)]
+        outs = [torch.empty(Bn, w.n_q_heads, 128, dtype=torch.float32, device="cuda") for _ in range(steps)]
+        torch.cuda.synchronize()
+        for i in range(steps):
+            B.append(c, kd[:, S0 + i:S0 + i + 1].contiguous(), vd[:, S0 + i:S0 + i + 1].contiguous(), sps[i], perm_k=perm)
+            if sync:
+                torch.cuda.synchronize()
+            B.decode_attn(c, qd[i], lens[i], perm_k=perm, out=outs[i], workspace=ws)
+            if sync:
+                torch.cuda.synchronize()
+        torch.cuda.synchronize()
+        runs.append((c, outs))
+    assert B.device_status() == 0
+    for a, b in zip(runs[0][1], runs[1][1]):
+        assert torch.equal(a, b)
+    for name in ("k_mant", "k_exp", "v_mant", "v_exp"):
+        assert torch.equal(getattr(runs[0][0], name), getattr(runs[1][0], name)), name
+    oc = oracle_cache(oracle, k, v, w.dtype, w.block, p, 720, perm_k=host(perm))
+    ref = oracle.decode_attn(oc, W.to_oracle(qs[-1]), w.dtype, w.n_q_heads, [S0 + steps] * Bn, perm_k=host(perm))
+    assert rel_err(host(runs[0][1][-1]).astype(np.float64), ref) <= ATTN_TOL
+
+
 def test_bounded_wait_runs_out_and_context_survives(oracle):
     """The bounded barrier wait of the staged kernels: a barrier whose bytes never arrive makes the wait give up after
     its tries, the kernel returns with KVBFP_FLAG_WAIT_TIMEOUT (and only that flag: the barrier whose bytes do arrive
