@@ -25,31 +25,53 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
     pdl_trigger();
     if (row >= n_rows) return;
     const int b = row / n_q_heads, hq = row % n_q_heads;
-    int len = seq_lens[b];
-    len = len < 0 ? 0 : (len > len_cap ? len_cap : len);
-    const int nc = (len + item_tokens - 1) / item_tokens;        // items that hold tokens
+    const int len_raw = seq_lens[b];        // (on its way while the slots are worked out and the partials asked for)
     const float* base = partials + (int64_t)row * n_chunks * kPartStride;
     const int first = (b * (n_q_heads / group) + hq / group) * items_per_pair;   // first item of the pair
-    // The partials of the row: with n_warps == 0 one per item; else one per range that holds items of the pair --
-    // the ranges are consecutive, and the k-th of them starts inside the pair at the first item of range w0 + k
-    // (the first one at item 0), so every lane finds its own partial without walking the others.
-    int w0 = 0, n_part = nc;
-    if (n_warps > 0 && nc > 0) {
+    // The partials of the row: with n_warps == 0 one per item that holds tokens; else one per range that holds such
+    // items of the pair -- the ranges are consecutive, and the k-th of them starts inside the pair at the first item
+    // of range w0 + k (the first one at item 0), so every lane finds its own partial without walking the others.
+    // Where the partials lie does not depend on the sequence's length, only how many of them there are: the loads
+    // go out for as many as the longest sequence allowed would have, and those beyond the real count are dropped
+    // unread (their slots hold whatever an earlier call left there).
+    const int nc_max = (len_cap + item_tokens - 1) / item_tokens;
+    int w0 = 0, n_part_max = nc_max;
+    if (n_warps > 0 && nc_max > 0) {
         w0 = range_of(first, range_items, range_extra);
-        n_part = range_of(first + nc - 1, range_items, range_extra) - w0 + 1;
+        n_part_max = range_of(first + nc_max - 1, range_items, range_extra) - w0 + 1;
     }
+    int n_part = -1;                         // known once the length has arrived
     float m = -INFINITY, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k0 = 0; k0 < n_part; k0 += 32) {
-        // a lane per partial: its slot, maximum and sum; then the weights of all 32 against the common maximum
+    for (int k0 = 0; k0 < n_part_max; k0 += 32) {
+        // a lane per partial: its slot, maximum and sum
         const int k = k0 + lane;
-        const bool have = k < n_part;
+        const bool may = k < n_part_max;
         int item = k;
-        if (n_warps > 0) item = max(range_start(w0 + (have ? k : 0), range_items, range_extra) - first, 0);
-        const int slot = have ? partial_slot(item, item_tokens, chunk, n_chunks) : 0;
+        if (n_warps > 0) item = max(range_start(w0 + (may ? k : 0), range_items, range_extra) - first, 0);
+        const int slot = may ? partial_slot(item, item_tokens, chunk, n_chunks) : 0;
         const float* pk = base + (int64_t)slot * kPartStride;
-        const float mk = have ? pk[D] : -INFINITY;
-        const float lk = have ? pk[D + 1] : 0.f;
+        const float mk_raw = may ? pk[D] : -INFINITY;
+        const float lk_raw = may ? pk[D + 1] : 0.f;
+        // the first eight vectors of this batch: every lane its four channels
+        float4 o0[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int sj = __shfl_sync(0xffffffffu, slot, u);
+            o0[u] = (k0 + u < n_part_max) ? *reinterpret_cast<const float4*>(base + (int64_t)sj * kPartStride + lane * 4)
+                                          : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        if (n_part < 0) {
+            const int len = len_raw < 0 ? 0 : (len_raw > len_cap ? len_cap : len_raw);
+            const int nc = (len + item_tokens - 1) / item_tokens;        // items that hold tokens
+            n_part = nc;
+            if (n_warps > 0 && nc > 0) n_part = range_of(first + nc - 1, range_items, range_extra) - w0 + 1;
+        }
+        if (k0 >= n_part) break;
+        // the weights of the batch against the common maximum
+        const bool have = k < n_part;
+        const float mk = have ? mk_raw : -INFINITY;
+        const float lk = have ? lk_raw : 0.f;
         float mn = mk;
 #pragma unroll
         for (int off = 16; off; off >>= 1) mn = fmaxf(mn, __shfl_xor_sync(0xffffffffu, mn, off));
@@ -62,16 +84,24 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
         acc.x *= a1; acc.y *= a1; acc.z *= a1; acc.w *= a1;
         l = l * a1 + ls;
         m = mn;
-        // the vectors, eight loads at a time: lane j's slot and weight go round, every lane adds its four channels
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const float aj = __shfl_sync(0xffffffffu, ak, u);              // 0 for lanes without a partial
+            if (aj != 0.f) {                                               // (a dropped slot may hold anything)
+                acc.x += aj * o0[u].x; acc.y += aj * o0[u].y; acc.z += aj * o0[u].z; acc.w += aj * o0[u].w;
+            }
+        }
+        // the rest of the batch, eight loads at a time: lane j's slot and weight go round
         const int cnt = min(32, n_part - k0);
-        for (int j0 = 0; j0 < cnt; j0 += 8) {
+        for (int j0 = 8; j0 < cnt; j0 += 8) {
             float4 oi[8];
             float aj[8];
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
                 const int sj = __shfl_sync(0xffffffffu, slot, (j0 + u) & 31);
                 aj[u] = __shfl_sync(0xffffffffu, ak, (j0 + u) & 31);       // 0 for lanes without a partial
-                oi[u] = *reinterpret_cast<const float4*>(base + (int64_t)sj * kPartStride + lane * 4);
+                oi[u] = (j0 + u < cnt) ? *reinterpret_cast<const float4*>(base + (int64_t)sj * kPartStride + lane * 4)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
             }
 #pragma unroll
             for (int u = 0; u < 8; ++u) {

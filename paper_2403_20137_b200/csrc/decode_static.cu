@@ -57,8 +57,9 @@ extern "C" kvbfp_status kvbfp_decode_attn_static(const kvbfp_cache* cache, const
     void* scratch = nullptr;
     st = scratch_address(&scratch);
     if (st != KVBFP_OK) return st;
-    // The workspace needs no initial contents: every partial result that the merge reads is written
-    // by this call first, so nothing has to be cleared between calls.
+    // The workspace needs no initial contents: every partial result that the merge uses is written by this call
+    // first (it may load slots beyond those before it knows the sequence's length, and drops them unused), so
+    // nothing has to be cleared between calls.
     return kvbfp_decode_attn(cache, q, q_dt, n_q_heads, seq_lens, max_len_hint, perm_k, inv_perm_v, softmax_scale,
                              q_mant_bits, out, scratch, kStaticScratchBytes, flags, stream);
 }
