@@ -273,8 +273,8 @@ def sweep_config5(B, dev):
         out[f"dequant_all_heads_{name}"] = {"tokens": T, "heads": H, "ms": ms, "GB/s": T * H * (68 + d * eb) / ms / 1e6}
     ms = timed(lambda: B.dequant_all(c, "k", T), reps=5)
     out["dequant_all_heads_f32_stored_order"] = {"tokens": T, "heads": H, "ms": ms, "GB/s": T * H * (68 + d * 4) / ms / 1e6}
-    _, _, inv = B.calibrate(k[0, :4096].contiguous(), H, d)
-    tabs = B.rope_tables(perm, inv, H, d, 10000.0, False, device=dev)
+    _, perm_r, inv_r = B.calibrate(k[0, :4096].contiguous(), H, d)      # (a permutation together with ITS inverse)
+    tabs = B.rope_tables(perm_r, inv_r, H, d, 10000.0, False, device=dev)
     rows = k[0]
     pos = torch.arange(T, dtype=torch.int32, device=dev)
     B.rope_apply(rows, pos, *tabs)
@@ -441,6 +441,8 @@ def main():
     ap.add_argument("--sweep5", action="store_true", help="(kept for old command lines: the sweep is part of the default run)")
     ap.add_argument("--no-sweep5", action="store_true", help="skip the prefill/append and calibration sweep (8 KV heads, 65536 "
                     "new tokens, blocks 16/32/64 x mantissas 4/6/8, calibration over 2^20 tokens, read-back paths) in the extras")
+    ap.add_argument("--sweep5-only", action="store_true", help="run that sweep alone and print its figures (a small case "
+                    "for profiling the cache-write, calibration, read-back and rotation kernels)")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
     over = {k: v for k, v in (("batch", args.batch), ("seq", args.seq), ("mant_bits", args.mant_bits),
@@ -461,6 +463,11 @@ def main():
     from paper_2403_20137_b200 import binding as B
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
+    if args.sweep5_only:
+        if rank == 0:
+            print(json.dumps({"workload": "config5 sweep: 8 KV heads x 128, 65536 new bf16 tokens, calibration over 2^20 tokens",
+                              "config5": sweep_config5(B, dev)}))
+        return
     dist = None
     if world > 1:
         import torch.distributed as dist
