@@ -1,16 +1,18 @@
 // Cache write: permute, shared exponent, round, clamp, pack, store (Sec. II-B last paragraph,
 // Sec. III par. 2 of the paper; Algorithm 1 step 3 applied at run time as a gather).
 //
-// Sixteen lanes own one (token, head) row of 128 channels, eight stored slots per lane; a thread block
-// takes sixteen tokens per step and each 16-lane group walks the heads of its token, so no index has to
-// be divided per row.  A block of n slots is held by n/8 neighbouring lanes; its largest magnitude is
-// found with xor-shuffles on the IEEE bit patterns (integer compare = exact).  Rounding to nearest-even
-// is one fused multiply-add with 1.5 * 2^23 + 2^(p-1): the integer M + 2^(p-1), which is the stored
-// field, appears in the low bits of the sum.
+// Sixteen lanes own one (token, head) row of 128 channels, eight stored slots per lane.  A block of n slots
+// is held by n/8 neighbouring lanes; its largest magnitude is found with xor-shuffles on the IEEE bit
+// patterns (integer compare = exact).  Rounding to nearest-even is one fused multiply-add with
+// 1.5 * 2^23 + 2^(p-1): the integer M + 2^(p-1), which is the stored field, appears in the low bits of
+// the sum.  Two kernels share this: append_quant_pack for single tokens (a thread block takes sixteen
+// tokens per step and each 16-lane group walks the heads of its token), append_rows for runs of tokens
+// (further down: a thread block per (sequence, head), rows staged through shared memory).
+#include <atomic>
+#include <type_traits>
+
 #include "common.cuh"
 #include "ptx.cuh"
-#include <type_traits>
-#include <atomic>
 
 namespace kvbfp {
 namespace {
