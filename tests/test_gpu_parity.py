@@ -626,6 +626,51 @@ def test_back_to_back_steps_equal_synchronised_steps(oracle, cfg, p):
     assert rel_err(host(runs[0][1][-1]).astype(np.float64), ref) <= ATTN_TOL
 
 
+def test_two_streams_interleaved_steps(oracle):
+    """Steps of two sequences' worth of work issued alternately on two streams (each stream its own cache, workspace
+    and outputs; the launches that overlap with their predecessors do so within their stream only) give what the same
+    steps give one stream after the other."""
+    w = W.CONFIGS[4]
+    Bn, S0, steps = 2, 400, 6
+    k, v = W.make_kv(w, n_tokens=S0 + steps, batch=Bn)
+    q0 = W.make_q(w, batch=Bn)
+    _, perm, _ = B.calibrate(dev(k.reshape(-1, w.n_kv_heads, 128)), w.n_kv_heads, 128)
+    z = dev(torch.zeros(Bn, dtype=torch.int32))
+    kd, vd = dev(k), dev(v)
+    results = []
+    for concurrent in (False, True):
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        rigs = []
+        for sidx in range(2):
+            c = B.Cache(Bn, w.n_kv_heads, 128, 416, w.block, w.mant_bits, fill=0)
+            B.append(c, kd[:, :S0].contiguous(), vd[:, :S0].contiguous(), z, perm_k=perm)
+            rigs.append({"cache": c,
+                         "ws": torch.empty(B.decode_workspace_bytes(c.fmt, w.n_q_heads), dtype=torch.uint8, device="cuda"),
+                         "q": [dev(torch.roll(q0, 3 * i + 7 * sidx, dims=-1)) for i in range(steps)],
+                         "outs": [torch.empty(Bn, w.n_q_heads, 128, dtype=torch.float32, device="cuda") for _ in range(steps)],
+                         "kn": [kd[:, S0 + i:S0 + i + 1].contiguous() for i in range(steps)],
+                         "vn": [vd[:, S0 + i:S0 + i + 1].contiguous() for i in range(steps)],
+                         "sp": [dev(torch.full((Bn,), S0 + i, dtype=torch.int32)) for i in range(steps)],
+                         "len": [dev(torch.full((Bn,), S0 + i + 1, dtype=torch.int32)) for i in range(steps)]})
+        torch.cuda.synchronize()
+        order = [(i, sidx) for i in range(steps) for sidx in range(2)] if concurrent else \
+                [(i, sidx) for sidx in range(2) for i in range(steps)]
+        for i, sidx in order:
+            r, st = rigs[sidx], streams[sidx]
+            B.append(r["cache"], r["kn"][i], r["vn"][i], r["sp"][i], perm_k=perm, stream=st)
+            B.decode_attn(r["cache"], r["q"][i], r["len"][i], perm_k=perm, out=r["outs"][i], workspace=r["ws"], stream=st)
+            if not concurrent:
+                st.synchronize()
+        torch.cuda.synchronize()
+        results.append(rigs)
+    assert B.device_status() == 0
+    for sidx in range(2):
+        for a, b in zip(results[0][sidx]["outs"], results[1][sidx]["outs"]):
+            assert torch.equal(a, b)
+        for name in ("k_mant", "k_exp", "v_mant", "v_exp"):
+            assert torch.equal(getattr(results[0][sidx]["cache"], name), getattr(results[1][sidx]["cache"], name)), name
+
+
 def test_bounded_wait_runs_out_and_context_survives(oracle):
     """The bounded barrier wait of the staged kernels: a barrier whose bytes never arrive makes the wait give up after
     its tries, the kernel returns with KVBFP_FLAG_WAIT_TIMEOUT (and only that flag: the barrier whose bytes do arrive
