@@ -12,6 +12,9 @@ namespace {
 // n_warps > 0: the items (pair-major pieces of item_tokens tokens) were cut into n_warps contiguous ranges and
 // each range wrote one partial per (batch, kv head) it touches, at the slot of the chunk in which its first
 // item there lies; the same integer arithmetic as in the kernel finds those slots.
+// SPLIT: a thread block per row, its four warps take every fourth partial and their results are merged through
+// shared memory (rows with many partials: long sequences cut into many ranges); else four rows per thread block.
+template <bool SPLIT>
 __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ partials, const int32_t* __restrict__ seq_lens,
                                                  const int32_t* __restrict__ inv_perm_v, float* __restrict__ out,
                                                  int n_rows, int n_q_heads, int group, int n_chunks, int chunk,
@@ -19,8 +22,9 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
                                                  int range_items, int range_extra) {
     constexpr int D = kHeadDim;
     __shared__ float so[4][D];
+    __shared__ float sml[4][2];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row = blockIdx.x * 4 + warp;           // b * Hq + hq
+    const int row = SPLIT ? blockIdx.x : blockIdx.x * 4 + warp;           // b * Hq + hq
     pdl_wait();
     pdl_trigger();
     if (row >= n_rows) return;
@@ -40,13 +44,17 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
         w0 = range_of(first, range_items, range_extra);
         n_part_max = range_of(first + nc_max - 1, range_items, range_extra) - w0 + 1;
     }
-    int n_part = -1;                         // known once the length has arrived
+    // this warp's share of them: all, or every fourth one starting at its own number
+    auto share = [&](int n) { return SPLIT ? (n > warp ? (n - warp + 3) >> 2 : 0) : n; };
+    const int n_sub_max = share(n_part_max);
+    int n_part = -1;                         // (of the warp's share) known once the length has arrived
     float m = -INFINITY, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int k0 = 0; k0 < n_part_max; k0 += 32) {
+    for (int k0 = 0; k0 < n_sub_max; k0 += 32) {
         // a lane per partial: its slot, maximum and sum
-        const int k = k0 + lane;
-        const bool may = k < n_part_max;
+        const int kk = k0 + lane;
+        const bool may = kk < n_sub_max;
+        const int k = SPLIT ? 4 * kk + warp : kk;
         int item = k;
         if (n_warps > 0) item = max(range_start(w0 + (may ? k : 0), range_items, range_extra) - first, 0);
         const int slot = may ? partial_slot(item, item_tokens, chunk, n_chunks) : 0;
@@ -58,7 +66,7 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int sj = __shfl_sync(0xffffffffu, slot, u);
-            o0[u] = (k0 + u < n_part_max) ? *reinterpret_cast<const float4*>(base + (int64_t)sj * kPartStride + lane * 4)
+            o0[u] = (k0 + u < n_sub_max) ? *reinterpret_cast<const float4*>(base + (int64_t)sj * kPartStride + lane * 4)
                                           : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         if (n_part < 0) {
@@ -66,10 +74,11 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
             const int nc = (len + item_tokens - 1) / item_tokens;        // items that hold tokens
             n_part = nc;
             if (n_warps > 0 && nc > 0) n_part = range_of(first + nc - 1, range_items, range_extra) - w0 + 1;
+            n_part = share(n_part);
         }
         if (k0 >= n_part) break;
         // the weights of the batch against the common maximum
-        const bool have = k < n_part;
+        const bool have = kk < n_part;
         const float mk = have ? mk_raw : -INFINITY;
         const float lk = have ? lk_raw : 0.f;
         float mn = mk;
@@ -108,6 +117,23 @@ __global__ void __launch_bounds__(128) lse_merge(const float* __restrict__ parti
                 acc.x += aj[u] * oi[u].x; acc.y += aj[u] * oi[u].y; acc.z += aj[u] * oi[u].z; acc.w += aj[u] * oi[u].w;
             }
         }
+    }
+    if (SPLIT) {       // the four warps' results into warp 0
+        *reinterpret_cast<float4*>(&so[warp][lane * 4]) = acc;
+        if (lane == 0) { sml[warp][0] = m; sml[warp][1] = l; }
+        __syncthreads();
+        if (warp != 0) return;
+        float mn = fmaxf(fmaxf(sml[0][0], sml[1][0]), fmaxf(sml[2][0], sml[3][0]));
+        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        l = 0.f;
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            const float a = (sml[w][0] == -INFINITY) ? 0.f : exp2f(sml[w][0] - mn);
+            const float4 o = *reinterpret_cast<const float4*>(&so[w][lane * 4]);
+            acc.x += a * o.x; acc.y += a * o.y; acc.z += a * o.z; acc.w += a * o.w;
+            l += a * sml[w][1];
+        }
+        __syncwarp();                                   // so[0] is reused below
     }
     const float inv = (l > 0.f) ? 1.f / l : 0.f;
     float* dst = out + (int64_t)row * D;
@@ -243,9 +269,18 @@ kvbfp_status decode_common(const kvbfp_cache* cache, const void* q, kvbfp_dtype 
     else st = launch_decode_mma(a, s);
     if (st != KVBFP_OK) return st;
     const int n_rows = f.batch * n_q_heads;
-    (void)launch_pdl(lse_merge, dim3((n_rows + 3) / 4), dim3(128), 0, s, (const float*)a.partials, seq_lens, inv_perm_v, out,
-                     n_rows, n_q_heads, group, a.n_chunks, a.chunk, a.len_cap, split.n_warps, split.item_tokens,
-                     split.items_per_pair, split.range_items, split.range_extra);
+    // partials per row, at most: a thread block per row where there are many (its warps share them)
+    const int per_row = split.n_warps > 0 ? (split.items_per_pair + (split.range_items > 0 ? split.range_items : 1) - 1) /
+                                                (split.range_items > 0 ? split.range_items : 1) + 1
+                                          : a.n_chunks;
+    if (per_row > 8)
+        (void)launch_pdl(lse_merge<true>, dim3(n_rows), dim3(128), 0, s, (const float*)a.partials, seq_lens, inv_perm_v, out,
+                         n_rows, n_q_heads, group, a.n_chunks, a.chunk, a.len_cap, split.n_warps, split.item_tokens,
+                         split.items_per_pair, split.range_items, split.range_extra);
+    else
+        (void)launch_pdl(lse_merge<false>, dim3((n_rows + 3) / 4), dim3(128), 0, s, (const float*)a.partials, seq_lens, inv_perm_v, out,
+                         n_rows, n_q_heads, group, a.n_chunks, a.chunk, a.len_cap, split.n_warps, split.item_tokens,
+                         split.items_per_pair, split.range_items, split.range_extra);
     KVBFP_LAUNCH_CHECK("lse_merge");
     return KVBFP_OK;
 }
