@@ -44,15 +44,15 @@ __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
         v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
     }
 }
-// Eight channels picked by the permutation, straight from the row (it sits in L1 after the first touch).
+// Eight channels picked by the permutation from the row parked in shared memory.
 __device__ __forceinline__ void gather8(const float* row, const int (&idx)[8], float (&v)[8]) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __ldg(row + idx[i]);
+    for (int i = 0; i < 8; ++i) v[i] = row[idx[i]];
 }
 __device__ __forceinline__ void gather8(const __nv_bfloat16* row, const int (&idx)[8], float (&v)[8]) {
 #pragma unroll
     for (int i = 0; i < 8; ++i)
-        v[i] = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(row) + idx[i]) << 16);
+        v[i] = __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(row)[idx[i]] << 16);
 }
 
 template <int P, int N, typename T>
@@ -72,6 +72,9 @@ __global__ void __launch_bounds__(kThreads) append_quant_pack(AppendArgs a) {
     const int32_t* perm = a.perm[which];
     const int sub = threadIdx.x & 15;          // lane within the row
     const int tloc = threadIdx.x >> 4;         // token within the thread block's step
+    // a permuted row is parked in shared memory by 16-byte loads that do not wait for the permutation, and picked
+    // apart from there (the gather straight from global memory was a second round trip behind the index loads)
+    __shared__ __align__(16) T srow[kTokPerCta][D];
     const int H = a.n_heads;
     const int64_t n_tok = (int64_t)a.batch * a.n_new;
 
@@ -95,7 +98,16 @@ __global__ void __launch_bounds__(kThreads) append_quant_pack(AppendArgs a) {
                 const int4 p0 = __ldg(pp), p1 = __ldg(pp + 1);
                 const int idx[8] = {p0.x & (D - 1), p0.y & (D - 1), p0.z & (D - 1), p0.w & (D - 1),
                                     p1.x & (D - 1), p1.y & (D - 1), p1.z & (D - 1), p1.w & (D - 1)};
-                gather8(tok + h * D, idx, v);
+                constexpr int VEC = 8 * (int)sizeof(T) / 16;            // 16-byte pieces of the lane's eight channels
+                const uint4* rp = reinterpret_cast<const uint4*>(tok + h * D + sub * 8);
+                uint4 raw[VEC];
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) raw[i] = __ldg(rp + i);
+                __syncwarp();                                   // the row parked before this one has been read
+#pragma unroll
+                for (int i = 0; i < VEC; ++i) reinterpret_cast<uint4*>(&srow[tloc][sub * 8])[i] = raw[i];
+                __syncwarp();
+                gather8(&srow[tloc][0], idx, v);
             } else {
                 load8(tok + h * D + sub * 8, v);
             }

@@ -215,6 +215,29 @@ def test_append_runs_ragged_tiles_and_nonfinite(oracle, dtype, p):
     assert bool((gb.v_mant == gc.v_mant).all())
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("p,n", [(4, 32), (6, 16), (8, 128), (4, 64)])
+def test_append_few_tokens_permuted_bit_exact(oracle, dtype, p, n):
+    """One, five and fifteen tokens per sequence (the kernel of the decode step's cache write), K and V permuted,
+    several sequences at different positions and more heads than one pass of a thread block takes: planes bit for bit."""
+    rng = np.random.default_rng(41)
+    H, Bn = 5, 3
+    perm_k = np.stack([rng.permutation(128) for _ in range(H)]).astype(np.int32)
+    perm_v = np.stack([rng.permutation(128) for _ in range(H)]).astype(np.int32)
+    base_k, base_v = adversarial_rows(dtype, seed=42), adversarial_rows(dtype, seed=43)      # [1, 96, 2, 128]
+    for T in (1, 5, 15):
+        k = base_k.reshape(3, 32, 2, 128).repeat(1, 1, 3, 1)[:, 7:7 + T, :H].contiguous()   # [3, T, H, 128]
+        v = base_v.reshape(3, 32, 2, 128).repeat(1, 1, 3, 1)[:, 11:11 + T, :H].contiguous()
+        start = [0, 9, 33]
+        gc = B.Cache(Bn, H, 128, 48, n, p, fill=0x3C)
+        B.append(gc, dev(k), dev(v), dev(torch.tensor(start, dtype=torch.int32)), dev(torch.from_numpy(perm_k)),
+                 dev(torch.from_numpy(perm_v)))
+        assert B.device_status() == 0
+        oc = oracle_cache(oracle, k, v, dtype, n, p, 48, start=start, perm_k=perm_k, perm_v=perm_v)
+        assert_planes_equal(gc, oc, [T] * Bn, start=start)
+        assert bool((gc.k_mant[1, :, :9] == 0x3C).all()) and bool((gc.v_exp[2, :, 33 + T:] == 0x3C).all())
+
+
 # ------------------------------------------------------------------------------- calibrate
 @pytest.mark.parametrize("cfg,T", [(1, 256), (2, 1000), (4, 777)])
 def test_calibrate_matches_oracle(oracle, cfg, T):
