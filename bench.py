@@ -38,7 +38,7 @@ UNIT = "tokens/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per (batch, kv head, token) unit on a smaller case of the
 # same kernel, scaled by the units of a launch.  Valid only while the kernel sources still hash to the
 # value recorded with the capture; otherwise the bench reports null.
-TRAFFIC = {"decode_mma4": {"bytes_per_unit": 137.8476, "block": 32, "mant_bits": 4, "sources_sha256": "ecc64b60e230c087cb94bf0c659446ca199cb23f695d105cc9aa88f8579bf878"},
+TRAFFIC = {"decode_mma4": {"bytes_per_unit": 138.2494, "block": 32, "mant_bits": 4, "sources_sha256": "3006fc386180fab06b257266496bbd0efb400e9c00028bf7c6fd405c7e93f5b1"},
            "decode_mma8": {"bytes_per_unit": 265.9599, "block": 32, "mant_bits": 8, "sources_sha256": "6ed4258b1fccf49c444f7130c499314796c7f5a30bf680a283449208da4f8c57"},
            "decode_mma6": {"bytes_per_unit": 201.705, "block": 32, "mant_bits": 6, "sources_sha256": "67627b858a3acb111ed91753e2373c139cfb0c3d831bb95f444c7884b64c04dc"}}
 KERNEL_SOURCES = {"decode_mma4": ["paper_2403_20137_b200/csrc/decode_mma4.cu", "paper_2403_20137_b200/csrc/ptx.cuh"],

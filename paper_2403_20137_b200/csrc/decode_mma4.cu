@@ -285,13 +285,47 @@ __global__ void __launch_bounds__(128) make_qfrag4i(DecodeArgs a, int NT, int32_
     if (item >= a.fmt.batch * a.fmt.n_kv_heads * NT) return;
     const int nt = item % NT, hk = (item / NT) % a.fmt.n_kv_heads, b = item / NT / a.fmt.n_kv_heads;
     const int Gq = a.n_q_heads / a.fmt.n_kv_heads;
+    // The four query rows of the n-tile are parked in shared memory by 16-byte loads that do not wait for the
+    // permutation's indices, and pi(q) is gathered from there (one memory round trip instead of two).
+    __shared__ __align__(16) float srow[4][4][D];                 // [warp][head of the n-tile][channel], raw bits
+    const int es = a.q_is_bf16 ? 2 : 4;
+    const int pieces = 4 * D * es / 16;                           // 16-byte pieces of the four rows: 64 or 128
+    uint8_t* park = reinterpret_cast<uint8_t*>(&srow[threadIdx.x >> 5][0][0]);
+    uint4 raw[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int pc = lane + 32 * i;                             // piece pc: head pc / (pieces / 4), piece of its row
+        raw[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (pc < pieces) {
+            const int hq = pc / (pieces / 4), off = pc % (pieces / 4);
+            const int qi = 4 * nt + hq;
+            if (qi < Gq)
+                raw[i] = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint8_t*>(a.q) +
+                                                              ((int64_t)b * a.n_q_heads + hk * Gq + qi) * D * es) + off);
+        }
+    }
     int ch[8];
     float qv[2][8];
     query_channels(a, hk, lane, ch);
 #pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int pc = lane + 32 * i;
+        if (pc < pieces) {
+            const int hq = pc / (pieces / 4), off = pc % (pieces / 4);
+            *reinterpret_cast<uint4*>(park + hq * (D * 4) + off * 16) = raw[i];     // (rows 512 bytes apart either way)
+        }
+    }
+    __syncwarp();
+#pragma unroll
     for (int pass = 0; pass < 2; ++pass) {
-        const int qi = 4 * nt + 2 * pass + (lane >> 4);
-        query_values(a, (int64_t)b * a.n_q_heads + hk * Gq + (qi < Gq ? qi : 0), qi < Gq, ch, qv[pass]);
+        const int hq = 2 * pass + (lane >> 4);
+        const uint8_t* row = park + hq * (D * 4);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int c = ch[j] & (D - 1);
+            qv[pass][j] = a.q_is_bf16 ? __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(row)[c] << 16)
+                                      : reinterpret_cast<const float*>(row)[c];
+        }
     }
     uint32_t qi8[8];
 #pragma unroll
